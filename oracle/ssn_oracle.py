@@ -1,0 +1,108 @@
+"""Plain CPU oracle for the subspace-network (SSN) stage-boundary codec.
+
+TEST INFRASTRUCTURE.  Only the tests, the smoke check and the benchmark's CPU-baseline leg may
+import this file.  It shares no code with the CUDA library and never calls it.
+
+Every function is the paper's definition written out in float64 with numpy; the only library
+primitive used as a step is a matrix product.  Nothing is blocked, fused or reordered.  Inputs
+are float64 arrays holding the exact values of the stored (fp32 / bf16) tensors; outputs are
+float64 and are not rounded.
+
+Notation (paper Sec. 4.1, "Pipeline-Parallel Communication with Reparameterized SSNs"):
+    X      [n, d]   hidden states, one row per token          (Eq. residual_stream)
+    U      [d, k]   orthonormal basis U_k of the shared subspace, used exactly as stored
+    E      [V, d]   fixed token embedding T_fixed; row ids[t] belongs to token t
+    P      [S, d]   positional embedding PE; row pos[t] belongs to token t
+    Z      [n, k]   the coordinates that cross the stage boundary   (Eq. ssn_compress)
+
+Readings taken where the text is silent (they are listed with their reasons in the design
+notes): the receiver adds E[ids] and P back after expanding with U^T; E and P are each
+optional; a token whose id or position is out of range takes a zero row for that term and
+raises a status bit instead of failing; the backward pass sends G U.
+
+Pins (tests/test_oracle_pins.py): hand-worked example, one-hot basis special case, bit-exact
+gather, isometry at k = d, exact round trip inside the subspace, adjoint and finite-difference
+identities, projector identities, explicit d x d projector, element-by-element loops on tiny
+shapes.  No function here is left unpinned.
+"""
+
+from __future__ import annotations
+
+from typing import Optional, Tuple
+
+import numpy as np
+
+STATUS_BAD_ID = 1
+STATUS_BAD_POS = 2
+
+
+def token_positions(n_tokens: int, seq_len: int) -> np.ndarray:
+    """Position of token t when a [batch, seq_len] batch is flattened batch-major."""
+    return np.arange(n_tokens, dtype=np.int64) % int(seq_len)
+
+
+def shift_rows(n_tokens: int, d: int, E: Optional[np.ndarray], ids: Optional[np.ndarray],
+               P: Optional[np.ndarray], pos: Optional[np.ndarray]) -> Tuple[np.ndarray, int]:
+    """The per-token shift T_fixed[ids[t]] + PE[pos[t]] of Eq. ssn_compress, and a status word.
+
+    A missing table contributes nothing.  An out-of-range index contributes a zero row and
+    sets STATUS_BAD_ID / STATUS_BAD_POS.
+    """
+    shift = np.zeros((n_tokens, d), dtype=np.float64)
+    status = 0
+    if E is not None:
+        ids = np.asarray(ids, dtype=np.int64)
+        ok = (ids >= 0) & (ids < E.shape[0])
+        if not ok.all():
+            status |= STATUS_BAD_ID
+        shift[ok] += np.asarray(E, dtype=np.float64)[ids[ok]]
+    if P is not None:
+        pos = np.asarray(pos, dtype=np.int64)
+        ok = (pos >= 0) & (pos < P.shape[0])
+        if not ok.all():
+            status |= STATUS_BAD_POS
+        shift[ok] += np.asarray(P, dtype=np.float64)[pos[ok]]
+    return shift, status
+
+
+def compress(X: np.ndarray, U: np.ndarray, E=None, ids=None, P=None, pos=None):
+    """Eq. ssn_compress: Z = (X - PE - T_fixed) U_k.  Returns (Z [n, k], status)."""
+    X = np.asarray(X, dtype=np.float64)
+    U = np.asarray(U, dtype=np.float64)
+    shift, status = shift_rows(X.shape[0], X.shape[1], E, ids, P, pos)
+    return (X - shift) @ U, status
+
+
+def decompress(Z: np.ndarray, U: np.ndarray, E=None, ids=None, P=None, pos=None):
+    """Receiver side of Eq. ssn_compress: Xhat = Z U_k^T + PE + T_fixed.  Returns (Xhat, status)."""
+    Z = np.asarray(Z, dtype=np.float64)
+    U = np.asarray(U, dtype=np.float64)
+    shift, status = shift_rows(Z.shape[0], U.shape[0], E, ids, P, pos)
+    return Z @ U.T + shift, status
+
+
+def grad_project_coeff(G: np.ndarray, U: np.ndarray) -> np.ndarray:
+    """Backward pass, "the same compression": the activation-gradient's coordinates dZ = G U_k."""
+    return np.asarray(G, dtype=np.float64) @ np.asarray(U, dtype=np.float64)
+
+
+def grad_project_full(G: np.ndarray, U: np.ndarray) -> np.ndarray:
+    """The projected gradient itself, G U_k U_k^T (coordinates kept unrounded in between)."""
+    U = np.asarray(U, dtype=np.float64)
+    return grad_project_coeff(G, U) @ U.T
+
+
+def weight_reproject(W: np.ndarray, U: np.ndarray, side: str) -> np.ndarray:
+    """Original-SSN step after each optimizer update: put an output projection back in span(U).
+
+    side = "right": W is [m, d] as in Eq. residual_stream (activations multiply it from the
+    left), its rows must lie in the subspace:  W <- (W U) U^T.
+    side = "left":  W is stored transposed, [d, m]:  W <- U (U^T W).
+    """
+    W = np.asarray(W, dtype=np.float64)
+    U = np.asarray(U, dtype=np.float64)
+    if side == "right":
+        return (W @ U) @ U.T
+    if side == "left":
+        return U @ (U.T @ W)
+    raise ValueError("side must be 'left' or 'right'")
