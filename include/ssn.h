@@ -1,0 +1,158 @@
+/*
+ * libssn -- subspace-network (SSN) stage-boundary codec for NVIDIA B200 (sm_100a).
+ *
+ * The four operations are the ones the Agora paper defines in Sec. 4.1 ("Pipeline-Parallel
+ * Communication with Reparameterized SSNs"); each declaration below cites the passage that
+ * defines it.  Notation: n tokens, model width d, subspace rank k,
+ *
+ *     X, G, Xhat  [n x d]   hidden states / activation-gradients, one row per token
+ *     Z, dZ       [n x k]   the coordinates that cross the stage boundary
+ *     U           [d x k]   orthonormal basis U_k of the shared subspace
+ *     E           [vocab x d]    fixed token embedding T_fixed (row ids[t] belongs to token t)
+ *     P           [max_pos x d]  positional embedding PE (row pos[t] belongs to token t)
+ *
+ * Common rules for every entry point
+ *   - All matrices are row-major with a leading dimension `ld*` counted in ELEMENTS
+ *     (ld >= number of columns).  One element type (`ssn_dtype_t`) is used for all of
+ *     X, G, Xhat, Z, dZ, W, U, E, P of a call; accumulation is always fp32.
+ *   - Every data pointer is a DEVICE pointer owned by the caller, except where a parameter is
+ *     explicitly called a host array.  The library never allocates, frees or synchronises;
+ *     each call only enqueues kernels on `stream` (a cudaStream_t passed as void*; NULL is
+ *     the default stream) and returns.
+ *   - The `ssn_codec_t` struct is read on the host during the call and may be discarded
+ *     afterwards; the device buffers it points to must stay valid until the enqueued work
+ *     has finished.
+ *   - Host-detectable mistakes (NULL pointer, k > d, ld too small, negative sizes, unknown
+ *     enum, workspace too small) return an error code before anything is launched.  A launch
+ *     the CUDA runtime rejects returns SSN_ERR_CUDA.  n_tokens == 0 (or batch == 0) is a
+ *     successful no-op.
+ *   - Device-detectable mistakes never trap: a token whose id is outside [0, vocab) or whose
+ *     position is outside [0, max_pos) takes a ZERO row for that term, and bit 0 (bad id) or
+ *     bit 1 (bad position) is OR-ed into *dev_status when that pointer is not NULL.  The
+ *     caller zeroes *dev_status beforehand.
+ *   - Inputs and outputs of one call must not overlap, except ssn_weight_reproject, which
+ *     works in place.
+ *   - bf16 buffers whose pointers are 16-byte aligned and whose leading dimensions are
+ *     multiples of 8 take the vectorised tensor-core kernels; anything else (fp32, odd
+ *     leading dimensions, unaligned views) is still computed, by slower general kernels.
+ */
+#ifndef SSN_H_
+#define SSN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SSN_VERSION 100
+
+typedef enum {
+  SSN_OK = 0,
+  SSN_ERR_NULL = 1,        /* a required pointer is NULL                                   */
+  SSN_ERR_SHAPE = 2,       /* a size, rank or leading dimension is impossible              */
+  SSN_ERR_DTYPE = 3,       /* unknown element type / side / mode                           */
+  SSN_ERR_WORKSPACE = 4,   /* workspace missing or smaller than the *_workspace_bytes size */
+  SSN_ERR_CUDA = 5         /* the CUDA runtime refused a launch                            */
+} ssn_status_t;
+
+typedef enum { SSN_F32 = 0, SSN_BF16 = 1 } ssn_dtype_t;
+
+/* Which side of W the subspace lives on (see ssn_weight_reproject). */
+typedef enum { SSN_SIDE_LEFT = 0, SSN_SIDE_RIGHT = 1 } ssn_side_t;
+
+/* What ssn_grad_project writes; the two may be OR-ed. */
+typedef enum { SSN_GRAD_COEFF = 1, SSN_GRAD_FULL = 2 } ssn_grad_mode_t;
+
+/* Bits of the device status word. */
+#define SSN_DEV_BAD_ID 1
+#define SSN_DEV_BAD_POS 2
+
+/*
+ * The data both ends of a stage boundary share (Sec. 4.1: the basis U_k, and PE and T_fixed
+ * "available to both sender and receiver").  Plain value struct; nothing is owned.
+ */
+typedef struct ssn_codec {
+  int32_t d;            /* model width, >= 1                                              */
+  int32_t k;            /* subspace rank, 1 <= k <= d                                     */
+  int32_t dtype;        /* ssn_dtype_t of every matrix                                    */
+  int32_t max_pos;      /* rows of P (ignored when P is NULL)                             */
+  const void *U;        /* device [d x k], required                                       */
+  int64_t ldu;          /* >= k                                                           */
+  const void *E;        /* device [vocab x d] or NULL: no token-embedding term            */
+  int64_t lde;          /* >= d                                                           */
+  int64_t vocab;        /* rows of E (ignored when E is NULL)                             */
+  const void *P;        /* device [max_pos x d] or NULL: no positional term (RoPE models) */
+  int64_t ldp;          /* >= d                                                           */
+} ssn_codec_t;
+
+/*
+ * Sender side, Eq. (ssn_compress):  Z[t,:] = (X[t,:] - P[pos(t),:] - E[ids[t],:]) U.
+ *   X     device [n_tokens x d], ldx >= d.
+ *   ids   device int32[n_tokens]; required when codec->E is not NULL, ignored otherwise.
+ *   pos   device int32[n_tokens] or NULL; NULL means pos(t) = t mod seq_len, the position of
+ *         token t in a batch-major [batch x seq_len] flattening (seq_len >= 1 required then).
+ *   Z     device [n_tokens x k] output, ldz >= k, rounded to the element type from fp32.
+ *   dev_status  device int32 or NULL (see the common rules).
+ */
+ssn_status_t ssn_compress(const ssn_codec_t *codec, const void *X, int64_t ldx,
+                          const int32_t *ids, const int32_t *pos, int64_t n_tokens,
+                          int32_t seq_len, void *Z, int64_t ldz, int32_t *dev_status,
+                          void *stream);
+
+/*
+ * Receiver side of Eq. (ssn_compress) ("the receiver reconstructs with U_k^T", and adds back
+ * the PE and T_fixed it also holds):  Xhat[t,:] = Z[t,:] U^T + E[ids[t],:] + P[pos(t),:].
+ * With codec->E == NULL and codec->P == NULL this is the plain expansion Z U^T, which is also
+ * how a receiving stage expands an incoming coefficient gradient.
+ * Arguments as for ssn_compress with Z the input and Xhat [n_tokens x d] the output.
+ */
+ssn_status_t ssn_decompress(const ssn_codec_t *codec, const void *Z, int64_t ldz,
+                            const int32_t *ids, const int32_t *pos, int64_t n_tokens,
+                            int32_t seq_len, void *Xhat, int64_t ldx, int32_t *dev_status,
+                            void *stream);
+
+/*
+ * Backward pass ("the backward pass uses the same compression"; chain rule (grad L) U_k):
+ *   mode & SSN_GRAD_COEFF:  dZ   [n_tokens x k] = G U           -- what crosses the link
+ *   mode & SSN_GRAD_FULL :  Gpar [n_tokens x d] = (G U) U^T     -- the projected gradient
+ * The coordinates are kept in fp32 between the two products of the FULL form.  E and P of the
+ * codec are not used.  dZ / Gpar may be NULL when their mode bit is clear.
+ */
+ssn_status_t ssn_grad_project(const ssn_codec_t *codec, const void *G, int64_t ldg,
+                              int64_t n_tokens, int32_t mode, void *dZ, int64_t ldz,
+                              void *Gpar, int64_t ldgp, void *stream);
+
+/*
+ * Original-SSN weight re-projection ("projecting it back into the subspace after every
+ * optimizer step", Sec. 4.1; done outside the autograd graph, ablation Sec. "Reparameterized
+ * SSN"), in place, for a batch of equally shaped weights:
+ *   SSN_SIDE_RIGHT: W is [rows x cols] with cols == d, the layout of Eq. (residual_stream)
+ *                   whose ROWS must lie in span(U):      W <- (W U) U^T
+ *   SSN_SIDE_LEFT : W is [rows x cols] with rows == d (the transposed storage):
+ *                                                        W <- U (U^T W)
+ *   W_ptrs   HOST array of `batch` device pointers, each [rows x cols] with leading
+ *            dimension ldw >= cols; the weights must be distinct buffers.
+ *   workspace  device scratch of at least ssn_weight_reproject_workspace_bytes(...) bytes,
+ *              16-byte aligned; may be NULL only when that size is 0.  Its contents are
+ *              garbage afterwards; calls that share it must be ordered on one stream.
+ * The k coordinates are kept in fp32 between the two products.
+ */
+size_t ssn_weight_reproject_workspace_bytes(const ssn_codec_t *codec, int64_t rows,
+                                            int64_t cols, int32_t side, int32_t batch);
+
+ssn_status_t ssn_weight_reproject(const ssn_codec_t *codec, void *const *W_ptrs, int32_t batch,
+                                  int64_t rows, int64_t cols, int64_t ldw, int32_t side,
+                                  void *workspace, size_t workspace_bytes, void *stream);
+
+/* Static, never-NULL description of a status code. */
+const char *ssn_status_string(ssn_status_t status);
+
+/* SSN_VERSION the library was built from. */
+int32_t ssn_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SSN_H_ */

@@ -1,0 +1,145 @@
+"""ctypes binding of libssn: the same names as the C-ABI, argument marshalling only.
+
+Every function takes raw device addresses (``tensor.data_ptr()``), sizes and a stream handle
+(``torch.cuda.current_stream().cuda_stream``) and forwards them; all arithmetic happens in the
+library's kernels.  Importing this module loads ``libssn.so`` from the package directory and
+raises ``ImportError`` if it has not been built -- there is no CPU fallback.
+"""
+
+from __future__ import annotations
+
+import ctypes
+import os
+import re
+from typing import Optional, Sequence
+
+from . import buildlib
+
+SSN_OK = 0
+SSN_ERR_NULL, SSN_ERR_SHAPE, SSN_ERR_DTYPE, SSN_ERR_WORKSPACE, SSN_ERR_CUDA = 1, 2, 3, 4, 5
+SSN_F32, SSN_BF16 = 0, 1
+SSN_SIDE_LEFT, SSN_SIDE_RIGHT = 0, 1
+SSN_GRAD_COEFF, SSN_GRAD_FULL = 1, 2
+SSN_DEV_BAD_ID, SSN_DEV_BAD_POS = 1, 2
+
+DTYPES = {"f32": SSN_F32, "bf16": SSN_BF16}
+SIDES = {"left": SSN_SIDE_LEFT, "right": SSN_SIDE_RIGHT}
+
+
+class SsnError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} (status {status})")
+
+
+class ssn_codec_t(ctypes.Structure):
+    _fields_ = [
+        ("d", ctypes.c_int32), ("k", ctypes.c_int32), ("dtype", ctypes.c_int32),
+        ("max_pos", ctypes.c_int32),
+        ("U", ctypes.c_void_p), ("ldu", ctypes.c_int64),
+        ("E", ctypes.c_void_p), ("lde", ctypes.c_int64), ("vocab", ctypes.c_int64),
+        ("P", ctypes.c_void_p), ("ldp", ctypes.c_int64),
+    ]
+
+
+def _load() -> ctypes.CDLL:
+    path = buildlib.LIB_PATH
+    if not os.path.exists(path):
+        raise ImportError(
+            f"{path} is missing: build it with `python -c 'import __graft_entry__ as g; g.build()'` "
+            "(the SSN codec runs only through its CUDA library)")
+    return ctypes.CDLL(path)
+
+
+_lib = _load()
+LIB_PATH = buildlib.LIB_PATH
+
+_vp, _i64, _i32, _sz = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32, ctypes.c_size_t
+_codec_p = ctypes.POINTER(ssn_codec_t)
+_SIGNATURES = {
+    "ssn_compress": (_i32, [_codec_p, _vp, _i64, _vp, _vp, _i64, _i32, _vp, _i64, _vp, _vp]),
+    "ssn_decompress": (_i32, [_codec_p, _vp, _i64, _vp, _vp, _i64, _i32, _vp, _i64, _vp, _vp]),
+    "ssn_grad_project": (_i32, [_codec_p, _vp, _i64, _i64, _i32, _vp, _i64, _vp, _i64, _vp]),
+    "ssn_weight_reproject_workspace_bytes": (_sz, [_codec_p, _i64, _i64, _i32, _i32]),
+    "ssn_weight_reproject": (_i32, [_codec_p, ctypes.POINTER(_vp), _i32, _i64, _i64, _i64, _i32,
+                                    _vp, _sz, _vp]),
+    "ssn_status_string": (ctypes.c_char_p, [_i32]),
+    "ssn_version": (_i32, []),
+}
+for _name, (_res, _args) in _SIGNATURES.items():
+    _fn = getattr(_lib, _name)
+    _fn.restype, _fn.argtypes = _res, _args
+
+
+def declared_symbols(header_dir: Optional[str] = None):
+    """Names of the functions the public headers declare (parsed from include/*.h)."""
+    header_dir = header_dir or os.path.join(buildlib.ROOT, "include")
+    names = []
+    for fname in sorted(os.listdir(header_dir)):
+        if fname.endswith(".h"):
+            text = open(os.path.join(header_dir, fname)).read()
+            text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+            names += re.findall(r"\b(ssn_[a-z0-9_]+)\s*\(", text)
+    return sorted(set(names))
+
+
+def status_string(status: int) -> str:
+    return _lib.ssn_status_string(int(status)).decode()
+
+
+def version() -> int:
+    return int(_lib.ssn_version())
+
+
+def make_codec(d: int, k: int, dtype: int, U: int, ldu: Optional[int] = None, E: int = 0,
+               lde: Optional[int] = None, vocab: int = 0, P: int = 0,
+               ldp: Optional[int] = None, max_pos: int = 0) -> ssn_codec_t:
+    """Fill an ``ssn_codec_t`` from raw device addresses (0 = NULL = term absent)."""
+    return ssn_codec_t(d=d, k=k, dtype=dtype, max_pos=max_pos, U=U or None,
+                       ldu=k if ldu is None else ldu, E=E or None,
+                       lde=d if lde is None else lde, vocab=vocab, P=P or None,
+                       ldp=d if ldp is None else ldp)
+
+
+def _check(status: int, where: str) -> None:
+    if status != SSN_OK:
+        raise SsnError(status, where)
+
+
+def ssn_compress(codec: ssn_codec_t, X: int, ldx: int, ids: int, pos: int, n_tokens: int,
+                 seq_len: int, Z: int, ldz: int, dev_status: int = 0, stream: int = 0) -> None:
+    _check(_lib.ssn_compress(ctypes.byref(codec), X or None, ldx, ids or None, pos or None,
+                             n_tokens, seq_len, Z or None, ldz, dev_status or None,
+                             stream or None), "ssn_compress")
+
+
+def ssn_decompress(codec: ssn_codec_t, Z: int, ldz: int, ids: int, pos: int, n_tokens: int,
+                   seq_len: int, Xhat: int, ldx: int, dev_status: int = 0, stream: int = 0) -> None:
+    _check(_lib.ssn_decompress(ctypes.byref(codec), Z or None, ldz, ids or None, pos or None,
+                               n_tokens, seq_len, Xhat or None, ldx, dev_status or None,
+                               stream or None), "ssn_decompress")
+
+
+def ssn_grad_project(codec: ssn_codec_t, G: int, ldg: int, n_tokens: int, mode: int, dZ: int = 0,
+                     ldz: int = 0, Gpar: int = 0, ldgp: int = 0, stream: int = 0) -> None:
+    _check(_lib.ssn_grad_project(ctypes.byref(codec), G or None, ldg, n_tokens, mode, dZ or None,
+                                 ldz, Gpar or None, ldgp, stream or None), "ssn_grad_project")
+
+
+def ssn_weight_reproject_workspace_bytes(codec: ssn_codec_t, rows: int, cols: int, side: int,
+                                         batch: int) -> int:
+    return int(_lib.ssn_weight_reproject_workspace_bytes(ctypes.byref(codec), rows, cols, side, batch))
+
+
+def ssn_weight_reproject(codec: ssn_codec_t, W_ptrs: Sequence[int], rows: int, cols: int, ldw: int,
+                         side: int, workspace: int = 0, workspace_bytes: int = 0,
+                         stream: int = 0) -> None:
+    arr = (_vp * max(1, len(W_ptrs)))(*[p or None for p in W_ptrs])
+    _check(_lib.ssn_weight_reproject(ctypes.byref(codec), arr, len(W_ptrs), rows, cols, ldw, side,
+                                     workspace or None, workspace_bytes, stream or None),
+           "ssn_weight_reproject")
+
+
+def raw(name: str):
+    """The raw ctypes function (returns the status instead of raising); used by error tests."""
+    return getattr(_lib, name)

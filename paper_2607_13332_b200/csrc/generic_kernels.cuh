@@ -1,0 +1,147 @@
+// General kernels of libssn: any element type, any rank, any leading dimension or alignment.
+// They are the fp32 path and the fallback for shapes the tensor-core kernels do not take.
+// Plain fp32 FMAs; one warp owns one token (or one row of W) and reduces over d with shuffles.
+#pragma once
+
+#include "ssn_common.cuh"
+
+namespace ssn {
+
+struct TokenArgs {
+  const void *src;   // [n x d] rows to project (X, G or W), or nullptr: read coordinates from zin
+  const void *zin;   // [n x k] coordinates when src == nullptr
+  void *zout;        // [n x k] coordinates out, nullable
+  void *dst;         // [n x d] expansion out, nullable (may alias src row-for-row)
+  const void *U;
+  int64_t lds, ldzin, ldzout, lddst, ldu;
+  int64_t n;
+  int32_t d, k;
+  int32_t sub_shift;  // phase 1 subtracts E[ids]+P[pos]   (Eq. ssn_compress)
+  int32_t add_shift;  // phase 2 adds E[ids]+P[pos] back   (receiver side)
+  ShiftTables shift;
+};
+
+constexpr int kGenericWarps = 8;
+constexpr int kGenericKChunk = 8;
+
+template <typename T>
+__global__ void __launch_bounds__(kGenericWarps * 32)
+token_kernel(const TokenArgs a) {
+  extern __shared__ float zs_all[];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int64_t t = (int64_t)blockIdx.x * kGenericWarps + warp;
+  if (t >= a.n) return;
+  float *zs = zs_all + (size_t)warp * a.k;
+  const T *U = static_cast<const T *>(a.U);
+
+  const T *erow = nullptr, *prow = nullptr;
+  if (a.sub_shift || a.add_shift) {
+    int64_t er = embedding_row(a.shift, t), pr = position_row(a.shift, t);
+    if (er >= 0) erow = static_cast<const T *>(a.shift.E) + er * a.shift.lde;
+    if (pr >= 0) prow = static_cast<const T *>(a.shift.P) + pr * a.shift.ldp;
+  }
+
+  if (a.src != nullptr) {
+    const T *x = static_cast<const T *>(a.src) + t * a.lds;
+    for (int j0 = 0; j0 < a.k; j0 += kGenericKChunk) {
+      float acc[kGenericKChunk];
+#pragma unroll
+      for (int jj = 0; jj < kGenericKChunk; ++jj) acc[jj] = 0.f;
+      const int jn = min(kGenericKChunk, a.k - j0);
+      for (int i = lane; i < a.d; i += 32) {
+        float r = to_f32(x[i]);
+        if (a.sub_shift) {
+          if (erow) r -= to_f32(erow[i]);
+          if (prow) r -= to_f32(prow[i]);
+        }
+        const T *urow = U + (int64_t)i * a.ldu + j0;
+#pragma unroll
+        for (int jj = 0; jj < kGenericKChunk; ++jj)
+          if (jj < jn) acc[jj] = fmaf(r, to_f32(urow[jj]), acc[jj]);
+      }
+#pragma unroll
+      for (int jj = 0; jj < kGenericKChunk; ++jj) {
+        float v = acc[jj];
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
+        if (lane == 0 && jj < jn) zs[j0 + jj] = v;
+      }
+    }
+    __syncwarp();
+    if (a.zout != nullptr) {
+      T *z = static_cast<T *>(a.zout) + t * a.ldzout;
+      for (int j = lane; j < a.k; j += 32) z[j] = from_f32<T>(zs[j]);
+    }
+  } else {
+    const T *z = static_cast<const T *>(a.zin) + t * a.ldzin;
+    for (int j = lane; j < a.k; j += 32) zs[j] = to_f32(z[j]);
+    __syncwarp();
+  }
+
+  if (a.dst != nullptr) {
+    T *out = static_cast<T *>(a.dst) + t * a.lddst;
+    for (int i = lane; i < a.d; i += 32) {
+      const T *urow = U + (int64_t)i * a.ldu;
+      float acc = 0.f;
+      for (int j = 0; j < a.k; ++j) acc = fmaf(zs[j], to_f32(urow[j]), acc);
+      if (a.add_shift) {
+        if (erow) acc += to_f32(erow[i]);
+        if (prow) acc += to_f32(prow[i]);
+      }
+      out[i] = from_f32<T>(acc);
+    }
+  }
+}
+
+// ---- LEFT re-projection, W [d x m]:  T = U^T W  then  W = U T ------------------------------
+struct LeftArgs {
+  void *W;          // [d x m]
+  const void *U;    // [d x k]
+  float *T;         // [k x m] fp32 scratch
+  int64_t ldw, ldu, m;
+  int32_t d, k;
+};
+
+constexpr int kLeftCols = 128;
+
+// T[j][c] = sum_i U[i][j] W[i][c]; thread = column c, blockIdx.y = chunk of 8 coordinates.
+template <typename T>
+__global__ void __launch_bounds__(kLeftCols) left_reduce_kernel(const LeftArgs a) {
+  const int64_t c = (int64_t)blockIdx.x * kLeftCols + threadIdx.x;
+  const int j0 = blockIdx.y * kGenericKChunk;
+  const int jn = min(kGenericKChunk, a.k - j0);
+  if (c >= a.m) return;
+  const T *W = static_cast<const T *>(a.W);
+  const T *U = static_cast<const T *>(a.U);
+  float acc[kGenericKChunk];
+#pragma unroll
+  for (int jj = 0; jj < kGenericKChunk; ++jj) acc[jj] = 0.f;
+  for (int i = 0; i < a.d; ++i) {
+    const float w = to_f32(W[(int64_t)i * a.ldw + c]);
+    const T *urow = U + (int64_t)i * a.ldu + j0;
+#pragma unroll
+    for (int jj = 0; jj < kGenericKChunk; ++jj)
+      if (jj < jn) acc[jj] = fmaf(to_f32(urow[jj]), w, acc[jj]);
+  }
+#pragma unroll
+  for (int jj = 0; jj < kGenericKChunk; ++jj)
+    if (jj < jn) a.T[(int64_t)(j0 + jj) * a.m + c] = acc[jj];
+}
+
+// W[i][c] = sum_j U[i][j] T[j][c]; thread = column c, blockIdx.y = block of 32 rows.
+template <typename T>
+__global__ void __launch_bounds__(kLeftCols) left_expand_kernel(const LeftArgs a) {
+  const int64_t c = (int64_t)blockIdx.x * kLeftCols + threadIdx.x;
+  if (c >= a.m) return;
+  T *W = static_cast<T *>(a.W);
+  const T *U = static_cast<const T *>(a.U);
+  const int i0 = blockIdx.y * 32, i1 = min(a.d, i0 + 32);
+  for (int i = i0; i < i1; ++i) {
+    const T *urow = U + (int64_t)i * a.ldu;
+    float acc = 0.f;
+    for (int j = 0; j < a.k; ++j) acc = fmaf(to_f32(urow[j]), a.T[(int64_t)j * a.m + c], acc);
+    W[(int64_t)i * a.ldw + c] = from_f32<T>(acc);
+  }
+}
+
+}  // namespace ssn

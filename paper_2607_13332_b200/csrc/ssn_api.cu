@@ -1,0 +1,250 @@
+// C-ABI of libssn: argument validation and kernel dispatch.  See include/ssn.h for the
+// contract of every entry point.
+#include "ssn.h"
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include "generic_kernels.cuh"
+#include "ssn_common.cuh"
+
+namespace ssn {
+namespace {
+
+inline bool valid_dtype(int32_t dt) { return dt == SSN_F32 || dt == SSN_BF16; }
+
+ssn_status_t check_codec(const ssn_codec_t *c) {
+  if (c == nullptr || c->U == nullptr) return SSN_ERR_NULL;
+  if (!valid_dtype(c->dtype)) return SSN_ERR_DTYPE;
+  if (c->d < 1 || c->k < 1 || c->k > c->d || c->ldu < c->k) return SSN_ERR_SHAPE;
+  return SSN_OK;
+}
+
+// Checks the shared tables when a call uses them and fills the device-side view.
+ssn_status_t make_shift(const ssn_codec_t *c, const int32_t *ids, const int32_t *pos,
+                        int32_t seq_len, int32_t *dev_status, ShiftTables *out) {
+  ShiftTables s{};
+  s.E = c->E;
+  s.P = c->P;
+  s.ids = ids;
+  s.pos = pos;
+  s.lde = c->lde;
+  s.ldp = c->ldp;
+  s.vocab = c->vocab;
+  s.max_pos = c->max_pos;
+  s.seq_len = seq_len;
+  s.dev_status = dev_status;
+  if (c->E != nullptr) {
+    if (ids == nullptr) return SSN_ERR_NULL;
+    if (c->lde < c->d || c->vocab < 1) return SSN_ERR_SHAPE;
+  }
+  if (c->P != nullptr) {
+    if (c->ldp < c->d || c->max_pos < 1) return SSN_ERR_SHAPE;
+    if (pos == nullptr && seq_len < 1) return SSN_ERR_SHAPE;
+  }
+  *out = s;
+  return SSN_OK;
+}
+
+ssn_status_t launch_status() {
+  return cudaGetLastError() == cudaSuccess ? SSN_OK : SSN_ERR_CUDA;
+}
+
+ssn_status_t launch_token_kernel(const TokenArgs &a, int32_t dtype, cudaStream_t stream) {
+  if (a.n == 0) return SSN_OK;
+  const int64_t blocks = (a.n + kGenericWarps - 1) / kGenericWarps;
+  if (blocks > 0x7fffffffLL) return SSN_ERR_SHAPE;
+  const size_t smem = (size_t)kGenericWarps * a.k * sizeof(float);
+  if (smem > 48 * 1024) {
+    cudaError_t e;
+    if (dtype == SSN_F32)
+      e = cudaFuncSetAttribute(token_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               (int)smem);
+    else
+      e = cudaFuncSetAttribute(token_kernel<__nv_bfloat16>,
+                               cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) {
+      cudaGetLastError();
+      return SSN_ERR_SHAPE;  // rank too large for the general kernel's shared memory
+    }
+  }
+  if (dtype == SSN_F32)
+    token_kernel<float><<<(unsigned)blocks, kGenericWarps * 32, smem, stream>>>(a);
+  else
+    token_kernel<__nv_bfloat16><<<(unsigned)blocks, kGenericWarps * 32, smem, stream>>>(a);
+  return launch_status();
+}
+
+}  // namespace
+}  // namespace ssn
+
+using namespace ssn;
+
+extern "C" {
+
+ssn_status_t ssn_compress(const ssn_codec_t *codec, const void *X, int64_t ldx,
+                          const int32_t *ids, const int32_t *pos, int64_t n_tokens,
+                          int32_t seq_len, void *Z, int64_t ldz, int32_t *dev_status,
+                          void *stream) {
+  ssn_status_t st = check_codec(codec);
+  if (st != SSN_OK) return st;
+  if (n_tokens < 0 || ldx < codec->d || ldz < codec->k) return SSN_ERR_SHAPE;
+  if (n_tokens == 0) return SSN_OK;
+  if (X == nullptr || Z == nullptr) return SSN_ERR_NULL;
+  TokenArgs a{};
+  st = make_shift(codec, ids, pos, seq_len, dev_status, &a.shift);
+  if (st != SSN_OK) return st;
+  a.src = X;
+  a.lds = ldx;
+  a.zout = Z;
+  a.ldzout = ldz;
+  a.U = codec->U;
+  a.ldu = codec->ldu;
+  a.n = n_tokens;
+  a.d = codec->d;
+  a.k = codec->k;
+  a.sub_shift = 1;
+  return launch_token_kernel(a, codec->dtype, static_cast<cudaStream_t>(stream));
+}
+
+ssn_status_t ssn_decompress(const ssn_codec_t *codec, const void *Z, int64_t ldz,
+                            const int32_t *ids, const int32_t *pos, int64_t n_tokens,
+                            int32_t seq_len, void *Xhat, int64_t ldx, int32_t *dev_status,
+                            void *stream) {
+  ssn_status_t st = check_codec(codec);
+  if (st != SSN_OK) return st;
+  if (n_tokens < 0 || ldx < codec->d || ldz < codec->k) return SSN_ERR_SHAPE;
+  if (n_tokens == 0) return SSN_OK;
+  if (Xhat == nullptr || Z == nullptr) return SSN_ERR_NULL;
+  TokenArgs a{};
+  st = make_shift(codec, ids, pos, seq_len, dev_status, &a.shift);
+  if (st != SSN_OK) return st;
+  a.zin = Z;
+  a.ldzin = ldz;
+  a.dst = Xhat;
+  a.lddst = ldx;
+  a.U = codec->U;
+  a.ldu = codec->ldu;
+  a.n = n_tokens;
+  a.d = codec->d;
+  a.k = codec->k;
+  a.add_shift = 1;
+  return launch_token_kernel(a, codec->dtype, static_cast<cudaStream_t>(stream));
+}
+
+ssn_status_t ssn_grad_project(const ssn_codec_t *codec, const void *G, int64_t ldg,
+                              int64_t n_tokens, int32_t mode, void *dZ, int64_t ldz,
+                              void *Gpar, int64_t ldgp, void *stream) {
+  ssn_status_t st = check_codec(codec);
+  if (st != SSN_OK) return st;
+  if ((mode & ~(SSN_GRAD_COEFF | SSN_GRAD_FULL)) != 0 || mode == 0) return SSN_ERR_DTYPE;
+  if (n_tokens < 0 || ldg < codec->d) return SSN_ERR_SHAPE;
+  if ((mode & SSN_GRAD_COEFF) && ldz < codec->k) return SSN_ERR_SHAPE;
+  if ((mode & SSN_GRAD_FULL) && ldgp < codec->d) return SSN_ERR_SHAPE;
+  if (n_tokens == 0) return SSN_OK;
+  if (G == nullptr) return SSN_ERR_NULL;
+  if ((mode & SSN_GRAD_COEFF) && dZ == nullptr) return SSN_ERR_NULL;
+  if ((mode & SSN_GRAD_FULL) && Gpar == nullptr) return SSN_ERR_NULL;
+  TokenArgs a{};
+  a.src = G;
+  a.lds = ldg;
+  if (mode & SSN_GRAD_COEFF) {
+    a.zout = dZ;
+    a.ldzout = ldz;
+  }
+  if (mode & SSN_GRAD_FULL) {
+    a.dst = Gpar;
+    a.lddst = ldgp;
+  }
+  a.U = codec->U;
+  a.ldu = codec->ldu;
+  a.n = n_tokens;
+  a.d = codec->d;
+  a.k = codec->k;
+  return launch_token_kernel(a, codec->dtype, static_cast<cudaStream_t>(stream));
+}
+
+size_t ssn_weight_reproject_workspace_bytes(const ssn_codec_t *codec, int64_t rows,
+                                            int64_t cols, int32_t side, int32_t batch) {
+  if (check_codec(codec) != SSN_OK || rows < 1 || cols < 1 || batch < 1) return 0;
+  if (side == SSN_SIDE_LEFT) return (size_t)codec->k * (size_t)cols * sizeof(float);
+  return 0;
+}
+
+ssn_status_t ssn_weight_reproject(const ssn_codec_t *codec, void *const *W_ptrs, int32_t batch,
+                                  int64_t rows, int64_t cols, int64_t ldw, int32_t side,
+                                  void *workspace, size_t workspace_bytes, void *stream) {
+  ssn_status_t st = check_codec(codec);
+  if (st != SSN_OK) return st;
+  if (side != SSN_SIDE_LEFT && side != SSN_SIDE_RIGHT) return SSN_ERR_DTYPE;
+  if (batch < 0 || rows < 1 || cols < 1 || ldw < cols) return SSN_ERR_SHAPE;
+  if ((side == SSN_SIDE_RIGHT ? cols : rows) != codec->d) return SSN_ERR_SHAPE;
+  if (batch == 0) return SSN_OK;
+  if (W_ptrs == nullptr) return SSN_ERR_NULL;
+  for (int32_t b = 0; b < batch; ++b)
+    if (W_ptrs[b] == nullptr) return SSN_ERR_NULL;
+  const size_t need = ssn_weight_reproject_workspace_bytes(codec, rows, cols, side, batch);
+  if (need > 0 && (workspace == nullptr || workspace_bytes < need)) return SSN_ERR_WORKSPACE;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+
+  if (side == SSN_SIDE_RIGHT) {
+    // Every row of W is one "token": project onto U and expand again, no shift terms.
+    for (int32_t b = 0; b < batch; ++b) {
+      TokenArgs a{};
+      a.src = W_ptrs[b];
+      a.lds = ldw;
+      a.dst = W_ptrs[b];
+      a.lddst = ldw;
+      a.U = codec->U;
+      a.ldu = codec->ldu;
+      a.n = rows;
+      a.d = codec->d;
+      a.k = codec->k;
+      st = launch_token_kernel(a, codec->dtype, s);
+      if (st != SSN_OK) return st;
+    }
+    return SSN_OK;
+  }
+
+  const int64_t col_blocks = (cols + kLeftCols - 1) / kLeftCols;
+  if (col_blocks > 0x7fffffffLL) return SSN_ERR_SHAPE;
+  for (int32_t b = 0; b < batch; ++b) {
+    LeftArgs a{};
+    a.W = W_ptrs[b];
+    a.U = codec->U;
+    a.T = static_cast<float *>(workspace);
+    a.ldw = ldw;
+    a.ldu = codec->ldu;
+    a.m = cols;
+    a.d = codec->d;
+    a.k = codec->k;
+    dim3 g1((unsigned)col_blocks, (unsigned)((codec->k + kGenericKChunk - 1) / kGenericKChunk));
+    dim3 g2((unsigned)col_blocks, (unsigned)((codec->d + 31) / 32));
+    if (codec->dtype == SSN_F32) {
+      left_reduce_kernel<float><<<g1, kLeftCols, 0, s>>>(a);
+      left_expand_kernel<float><<<g2, kLeftCols, 0, s>>>(a);
+    } else {
+      left_reduce_kernel<__nv_bfloat16><<<g1, kLeftCols, 0, s>>>(a);
+      left_expand_kernel<__nv_bfloat16><<<g2, kLeftCols, 0, s>>>(a);
+    }
+    st = launch_status();
+    if (st != SSN_OK) return st;
+  }
+  return SSN_OK;
+}
+
+const char *ssn_status_string(ssn_status_t status) {
+  switch (status) {
+    case SSN_OK: return "ok";
+    case SSN_ERR_NULL: return "a required pointer is NULL";
+    case SSN_ERR_SHAPE: return "impossible size, rank or leading dimension";
+    case SSN_ERR_DTYPE: return "unknown element type, side or mode";
+    case SSN_ERR_WORKSPACE: return "workspace missing or too small";
+    case SSN_ERR_CUDA: return "the CUDA runtime refused a launch";
+  }
+  return "unknown status";
+}
+
+int32_t ssn_version(void) { return SSN_VERSION; }
+
+}  // extern "C"

@@ -1,0 +1,127 @@
+"""Torch-tensor convenience layer over the ctypes binding.
+
+Torch is used for device memory and streams only: every method below allocates the output,
+hands raw addresses to the C-ABI call of the same name and returns.  No arithmetic happens in
+Python and nothing here works without the CUDA library.
+"""
+
+from __future__ import annotations
+
+from typing import List, Optional, Sequence
+
+import numpy as np
+import torch
+
+from . import binding, synth
+
+_TORCH_DTYPE = {synth.F32: torch.float32, synth.BF16: torch.bfloat16}
+
+
+def to_device(stored: Optional[np.ndarray], dtype: str, device: str = "cuda") -> Optional[torch.Tensor]:
+    """Upload a tensor kept in storage form (float32 array or uint16 bf16 bits)."""
+    if stored is None:
+        return None
+    if dtype == synth.F32:
+        return torch.from_numpy(np.ascontiguousarray(stored, dtype=np.float32)).to(device)
+    bits = np.ascontiguousarray(stored, dtype=np.uint16).view(np.int16)
+    return torch.from_numpy(bits).to(device).view(torch.bfloat16)
+
+
+def to_host(t: torch.Tensor, dtype: str) -> np.ndarray:
+    """Download to storage form (float32 array or uint16 bf16 bits)."""
+    if dtype == synth.F32:
+        return t.detach().cpu().numpy()
+    return t.detach().contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _ld(t: torch.Tensor) -> int:
+    if t.dim() != 2 or t.stride(1) != 1:
+        raise ValueError("expected a row-major 2-D tensor (unit stride along the last dimension)")
+    return t.stride(0) if t.shape[0] > 1 else max(t.stride(0), t.shape[1])
+
+
+class Codec:
+    """The data both ends of a stage boundary share: U [d,k], optional E [V,d] and P [S,d]."""
+
+    def __init__(self, dtype: str, U: torch.Tensor, E: Optional[torch.Tensor] = None,
+                 P: Optional[torch.Tensor] = None):
+        self.dtype = dtype
+        self.U, self.E, self.P = U, E, P
+        self.d, self.k = U.shape
+        for t in (U, E, P):
+            if t is not None and (not t.is_cuda or t.dtype != _TORCH_DTYPE[dtype]):
+                raise ValueError("codec tensors must be CUDA tensors of the codec dtype")
+        self.dev_status = torch.zeros(1, dtype=torch.int32, device=U.device)
+        self.c = binding.make_codec(
+            self.d, self.k, binding.DTYPES[dtype], U.data_ptr(), _ld(U),
+            E.data_ptr() if E is not None else 0, _ld(E) if E is not None else None,
+            E.shape[0] if E is not None else 0,
+            P.data_ptr() if P is not None else 0, _ld(P) if P is not None else None,
+            P.shape[0] if P is not None else 0)
+
+    def _empty(self, rows: int, cols: int) -> torch.Tensor:
+        return torch.empty((rows, cols), dtype=_TORCH_DTYPE[self.dtype], device=self.U.device)
+
+    def take_status(self) -> int:
+        """Read and clear the device status word (synchronises)."""
+        v = int(self.dev_status.item())
+        self.dev_status.zero_()
+        return v
+
+    def compress(self, X: torch.Tensor, ids: Optional[torch.Tensor] = None, seq_len: int = 1,
+                 pos: Optional[torch.Tensor] = None, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+        n = X.shape[0]
+        Z = out if out is not None else self._empty(n, self.k)
+        binding.ssn_compress(self.c, X.data_ptr(), _ld(X), ids.data_ptr() if ids is not None else 0,
+                             pos.data_ptr() if pos is not None else 0, n, seq_len, Z.data_ptr(),
+                             _ld(Z), self.dev_status.data_ptr(), _stream())
+        return Z
+
+    def decompress(self, Z: torch.Tensor, ids: Optional[torch.Tensor] = None, seq_len: int = 1,
+                   pos: Optional[torch.Tensor] = None, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+        n = Z.shape[0]
+        Xh = out if out is not None else self._empty(n, self.d)
+        binding.ssn_decompress(self.c, Z.data_ptr(), _ld(Z), ids.data_ptr() if ids is not None else 0,
+                               pos.data_ptr() if pos is not None else 0, n, seq_len, Xh.data_ptr(),
+                               _ld(Xh), self.dev_status.data_ptr(), _stream())
+        return Xh
+
+    def grad_project(self, G: torch.Tensor, full: bool = False, coeff: bool = True,
+                     out: Optional[torch.Tensor] = None, out_full: Optional[torch.Tensor] = None):
+        n = G.shape[0]
+        mode = (binding.SSN_GRAD_COEFF if coeff else 0) | (binding.SSN_GRAD_FULL if full else 0)
+        dZ = (out if out is not None else self._empty(n, self.k)) if coeff else None
+        Gp = (out_full if out_full is not None else self._empty(n, self.d)) if full else None
+        binding.ssn_grad_project(self.c, G.data_ptr(), _ld(G), n, mode,
+                                 dZ.data_ptr() if coeff else 0, _ld(dZ) if coeff else 0,
+                                 Gp.data_ptr() if full else 0, _ld(Gp) if full else 0, _stream())
+        if coeff and full:
+            return dZ, Gp
+        return dZ if coeff else Gp
+
+    def reproject_workspace(self, rows: int, cols: int, side: str, batch: int) -> Optional[torch.Tensor]:
+        nbytes = binding.ssn_weight_reproject_workspace_bytes(self.c, rows, cols, binding.SIDES[side], batch)
+        if nbytes == 0:
+            return None
+        return torch.empty(nbytes, dtype=torch.uint8, device=self.U.device)
+
+    def weight_reproject(self, weights: Sequence[torch.Tensor], side: str,
+                         workspace: Optional[torch.Tensor] = None) -> None:
+        """In place, for a list of equally shaped weights."""
+        if not weights:
+            return
+        rows, cols = weights[0].shape
+        ldw = _ld(weights[0])
+        for w in weights:
+            if tuple(w.shape) != (rows, cols) or _ld(w) != ldw:
+                raise ValueError("weights of one call must share shape and leading dimension")
+        if workspace is None:
+            workspace = self.reproject_workspace(rows, cols, side, len(weights))
+        binding.ssn_weight_reproject(self.c, [w.data_ptr() for w in weights], rows, cols, ldw,
+                                     binding.SIDES[side],
+                                     workspace.data_ptr() if workspace is not None else 0,
+                                     workspace.numel() if workspace is not None else 0, _stream())
