@@ -1,0 +1,366 @@
+#!/usr/bin/env python
+"""Benchmark of the SSN stage-boundary codec on B200.
+
+One *step* is one pass of the whole hot path over one microbatch of the 8B-class stage
+boundary (d=4096, k=40, vocab 128256, 32 x 2048 = 65536 tokens, bf16, Zipf(1.1) token ids):
+
+    compress  Z  = (X - E[ids] - P) U          (sender, forward)
+    decompress Xhat = Z U^T + E[ids] + P       (receiver, forward)
+    grad-project dZ = G U                      (backward)
+    weight re-projection W <- (W U) U^T of one transformer block's attention out-projection
+        [4096 x 4096] and MLP down-projection [14336 x 4096]   (after the optimizer step)
+
+The metric is tokens per second through that step.  Every rank runs its own replica on its own
+microbatch (tokens are independent, so there is no collective on the data path): weak scaling.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+`--impl reference` times the CPU oracle (test infrastructure, as it stands) on a bounded sample.
+"""
+
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "ssn_codec_tokens_per_s"
+UNIT = "tokens/s"
+FALLBACK_HBM_GBS = 6650.0
+
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of ONE launch of the dominant
+# kernel on this workload, from the ncu capture summarised under profiles/; None until captured.
+NCU_TRAFFIC_BYTES = {"compress": None}
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--batch", type=int, default=None, help="sequences per microbatch (default 32)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-seconds", type=float, default=12.0)
+    return ap.parse_args()
+
+
+def workload(args):
+    from paper_2607_13332_b200 import synth
+
+    wl = synth.STAGE_8B
+    if args.batch is not None:
+        wl = wl.scaled(batch=args.batch)
+    return wl
+
+
+def config_of(wl, world):
+    return {
+        "workload": f"8B-class stage boundary: d={wl.d}, k={wl.k}, vocab={wl.vocab}, "
+                    f"{wl.batch}x{wl.seq_len}={wl.n_tokens} tokens, bf16, Zipf({wl.zipf_s}) ids; "
+                    "compress + decompress + grad-project + re-projection of one block's "
+                    "out-proj [4096x4096] and down-proj [14336x4096] per step",
+        "d": wl.d, "k": wl.k, "vocab": wl.vocab, "tokens_per_rank": wl.n_tokens,
+        "replicas": world, "l2": "inputs larger than L2 (X, G, E: 0.5-1 GB each)",
+    }
+
+
+# ----------------------------------------------------------------------------------------------
+# compulsory ("algorithmic") bytes of one launch: each distinct table row counted once
+# ----------------------------------------------------------------------------------------------
+def algorithmic_bytes(wl, ids, step):
+    b = 2
+    n, d, k = wl.n_tokens, wl.d, wl.k
+    uniq = int(np.unique(ids).size)
+    shift = uniq * d * b + min(wl.seq_len, n) * d * b
+    if step in ("compress", "decompress"):
+        return n * d * b + shift + d * k * b + n * k * b
+    if step == "grad_project":
+        return n * d * b + d * k * b + n * k * b
+    raise ValueError(step)
+
+
+# ----------------------------------------------------------------------------------------------
+# CPU oracle leg (cpu_baseline of the GPU arm, and the whole of --impl reference)
+# ----------------------------------------------------------------------------------------------
+def oracle_tokens_per_s(wl, seconds, seed=0x5EED + 32):
+    """Times the oracle, as it stands, on a bounded sample of the step: `sample` tokens through
+    compress, decompress and grad-project plus the same fraction of the two weights' rows."""
+    from threadpoolctl import threadpool_info
+
+    from oracle import ssn_oracle as oracle
+    from paper_2607_13332_b200 import synth
+
+    sample = min(wl.n_tokens, 4096)
+    small = synth.Workload("sample", wl.d, wl.k, min(wl.vocab, 16384), 1, sample, wl.dtype,
+                           wl.ids_law, wl.zipf_s)
+    t = synth.codec_inputs(small, seed=seed)
+    pos = oracle.token_positions(sample, wl.seq_len)
+    P = synth.to_storage(synth.sinusoidal_positions(wl.seq_len, wl.d), wl.dtype)
+    w_rows = max(1, (4096 + 14336) * sample // wl.n_tokens)
+    W = synth.projection_weight(w_rows, wl.d, seed, wl.dtype)
+
+    f = lambda a: synth.to_f64(a, wl.dtype)
+    U, E, Pf = f(t["U"]), f(t["E"]), f(P)      # the shared tables are set up once, untimed
+
+    def one_pass():
+        Z, _ = oracle.compress(f(t["X"]), U, E, t["ids"], Pf, pos)
+        oracle.decompress(Z, U, E, t["ids"], Pf, pos)
+        oracle.grad_project_coeff(f(t["G"]), U)
+        oracle.weight_reproject(f(W), U, "right")
+
+    one_pass()
+    t0 = time.perf_counter()
+    one_pass()
+    per_pass = time.perf_counter() - t0
+    reps = max(1, int(seconds / max(per_pass, 1e-3)))
+    t0 = time.perf_counter()
+    for _ in range(reps):
+        one_pass()
+    elapsed = time.perf_counter() - t0
+    cores = max([i.get("num_threads", 1) for i in threadpool_info()] or [1])
+    return {
+        "value": sample * reps / elapsed, "unit": UNIT, "cores": int(cores), "kind": "oracle",
+        "sample": f"{reps} passes over {sample} tokens (+{w_rows} weight rows) of the step, "
+                  f"numpy fp64, {elapsed:.1f} s",
+    }, elapsed / reps
+
+
+# ----------------------------------------------------------------------------------------------
+# clocks during the timed region
+# ----------------------------------------------------------------------------------------------
+class ClockSampler:
+    QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+    NAMES = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+
+    def __init__(self, index: int):
+        self.lines = []
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
+                 "-lms", "100", "-i", str(index)], stdout=subprocess.PIPE, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append((time.perf_counter(), line.strip()))
+
+    def stop(self, t_begin=None, t_end=None):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        rows = [l for (ts, l) in self.lines if (t_begin is None or t_begin <= ts <= t_end + 0.1)]
+        if not rows:
+            rows = [l for (_, l) in self.lines]
+        sm, smax, reasons = [], [], set()
+        for row in rows:
+            parts = [p.strip() for p in row.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                smax.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, flag in zip(self.NAMES, parts[3:7]):
+                if flag.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None,
+                "sm_max_mhz": float(max(smax)) if smax else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def measured_hbm_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as fh:
+            return float(json.load(fh)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    except (OSError, KeyError, ValueError):
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+# ----------------------------------------------------------------------------------------------
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    wl = workload(args)
+    total_steps = args.warmup + args.steps
+    per_step_seconds = max(1.0, min(args.cpu_seconds, 120.0 / max(1, total_steps)))
+    values, last = [], None
+    for i in range(total_steps):
+        last, per_pass = oracle_tokens_per_s(wl, per_step_seconds)
+        if i >= args.warmup:
+            values.append(last["value"])
+    value = float(np.mean(values))
+    last["value"] = value
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * wl.n_tokens / value,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic", "config": config_of(wl, 1), "cpu_baseline": last,
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    import __graft_entry__ as entry
+    entry.build()
+    from paper_2607_13332_b200 import binding, synth
+    from paper_2607_13332_b200.runner import Codec, to_device
+
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the SSN codec has no CPU path")
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    wl = workload(args)
+    dt = wl.dtype
+    t = synth.codec_inputs(wl, seed=0x5EED + 32 + 1000 * rank)
+    codec = Codec(dt, to_device(t["U"], dt), to_device(t["E"], dt), to_device(t["P"], dt))
+    n, d, k = wl.n_tokens, wl.d, wl.k
+    ids_h = torch.from_numpy(t["ids"]).pin_memory()
+    X_h = torch.from_numpy(t["X"].view(np.int16)).view(torch.bfloat16).pin_memory()
+    G_h = torch.from_numpy(t["G"].view(np.int16)).view(torch.bfloat16).pin_memory()
+    X, G, ids = X_h.cuda(), G_h.cuda(), ids_h.cuda()
+    Z = torch.empty((n, k), dtype=torch.bfloat16, device="cuda")
+    dZ = torch.empty_like(Z)
+    Xh = torch.empty_like(X)
+    Z_h, dZ_h = Z.cpu().pin_memory(), dZ.cpu().pin_memory()
+    weights = [to_device(synth.projection_weight(r, c, 0x5EED, dt, layer=i), dt)
+               for i, (r, c) in enumerate(synth.REPROJECT_SHAPES_8B.values())]
+    groups = [[w] for w in weights]
+    work = [codec.reproject_workspace(w.shape[0], w.shape[1], "right", 1) for w in weights]
+    del t["X"], t["G"], t["E"]
+
+    stream = torch.cuda.current_stream()
+    kernel_events = []
+
+    def step(record=False):
+        if record:
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+        codec.compress(X, ids, seq_len=wl.seq_len, out=Z)
+        if record:
+            e1.record(stream)
+            kernel_events.append((e0, e1))
+        codec.decompress(Z, ids, seq_len=wl.seq_len, out=Xh)
+        codec.grad_project(G, out=dZ)
+        for g, ws in zip(groups, work):
+            codec.weight_reproject(g, "right", workspace=ws)
+
+    def e2e_step():
+        X.copy_(X_h, non_blocking=True)
+        G.copy_(G_h, non_blocking=True)
+        ids.copy_(ids_h, non_blocking=True)
+        step()
+        Z_h.copy_(Z, non_blocking=True)
+        dZ_h.copy_(dZ, non_blocking=True)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(fn, steps, **kw):
+        barrier()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for _ in range(steps):
+            fn(**kw)
+        b.record(stream)
+        barrier()
+        ms = torch.tensor([a.elapsed_time(b)], device="cuda")
+        if world > 1:
+            dist.all_reduce(ms, op=dist.ReduceOp.MAX)
+        return float(ms.item())
+
+    for _ in range(max(3, args.warmup)):
+        step()
+    sampler = ClockSampler(local) if rank == 0 else None
+    launches0 = binding.ssn_launch_count()
+    t_begin = time.perf_counter()
+    ms_total = timed(step, args.steps)
+    launches = binding.ssn_launch_count() - launches0
+    # same loop once more with events around the dominant kernel (events add small gaps, so
+    # this pass is not the one that gives `value`)
+    timed(step, args.steps, record=True)
+    t_end = time.perf_counter()
+    clocks = sampler.stop(t_begin, t_end) if sampler else None
+    compress_ms = float(np.mean([a.elapsed_time(b) for a, b in kernel_events]))
+    for _ in range(2):
+        e2e_step()
+    ms_e2e = timed(e2e_step, args.steps)
+    status = codec.take_status()
+    if status != 0:
+        raise RuntimeError(f"device status {status}: synthetic ids/positions out of range")
+
+    if rank == 0:
+        ms_per_step = ms_total / args.steps
+        value = world * n / (ms_per_step * 1e-3)
+        peak, peak_kind = measured_hbm_peak()
+        algo = algorithmic_bytes(wl, t["ids"], "compress")
+        achieved = algo / (compress_ms * 1e-3) / 1e9
+        h2d = X_h.numel() * 2 + G_h.numel() * 2 + ids_h.numel() * 4
+        d2h = Z_h.numel() * 2 + dZ_h.numel() * 2
+        out = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": config_of(wl, world),
+            "roofline": {"bound": "hbm", "kernel": "ssn_compress", "achieved": achieved,
+                         "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                         "peak_kind": peak_kind, "algorithmic_bytes": algo,
+                         "kernel_ms": compress_ms, "traffic": NCU_TRAFFIC_BYTES["compress"]},
+            "e2e": {"value": world * n / (ms_e2e / args.steps * 1e-3), "unit": UNIT,
+                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+            "gpu_launches": int(launches),
+            "clocks": clocks,
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            out["cpu_baseline"], _ = oracle_tokens_per_s(wl, args.cpu_seconds)
+        print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

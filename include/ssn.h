@@ -152,6 +152,13 @@ const char *ssn_status_string(ssn_status_t status);
 /* SSN_VERSION the library was built from. */
 int32_t ssn_version(void);
 
+/*
+ * Diagnostic: how many kernels this process has enqueued through the library so far (all
+ * entry points, all streams).  No counterpart in the paper; the benchmark uses it to report
+ * its launch count.
+ */
+int64_t ssn_launch_count(void);
+
 #ifdef __cplusplus
 }
 #endif

@@ -65,6 +65,7 @@ _SIGNATURES = {
                                     _vp, _sz, _vp]),
     "ssn_status_string": (ctypes.c_char_p, [_i32]),
     "ssn_version": (_i32, []),
+    "ssn_launch_count": (_i64, []),
 }
 for _name, (_res, _args) in _SIGNATURES.items():
     _fn = getattr(_lib, _name)
@@ -89,6 +90,10 @@ def status_string(status: int) -> str:
 
 def version() -> int:
     return int(_lib.ssn_version())
+
+
+def ssn_launch_count() -> int:
+    return int(_lib.ssn_launch_count())
 
 
 def make_codec(d: int, k: int, dtype: int, U: int, ldu: Optional[int] = None, E: int = 0,

@@ -5,6 +5,8 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
+#include <atomic>
+
 #include "generic_kernels.cuh"
 #include "ssn_common.cuh"
 
@@ -46,7 +48,11 @@ ssn_status_t make_shift(const ssn_codec_t *c, const int32_t *ids, const int32_t 
   return SSN_OK;
 }
 
-ssn_status_t launch_status() {
+std::atomic<int64_t> g_launches{0};
+
+// Called after every group of `launches` kernel launches.
+ssn_status_t launch_status(int launches = 1) {
+  g_launches.fetch_add(launches, std::memory_order_relaxed);
   return cudaGetLastError() == cudaSuccess ? SSN_OK : SSN_ERR_CUDA;
 }
 
@@ -227,7 +233,7 @@ ssn_status_t ssn_weight_reproject(const ssn_codec_t *codec, void *const *W_ptrs,
       left_reduce_kernel<__nv_bfloat16><<<g1, kLeftCols, 0, s>>>(a);
       left_expand_kernel<__nv_bfloat16><<<g2, kLeftCols, 0, s>>>(a);
     }
-    st = launch_status();
+    st = launch_status(2);
     if (st != SSN_OK) return st;
   }
   return SSN_OK;
@@ -246,5 +252,7 @@ const char *ssn_status_string(ssn_status_t status) {
 }
 
 int32_t ssn_version(void) { return SSN_VERSION; }
+
+int64_t ssn_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 }  // extern "C"
