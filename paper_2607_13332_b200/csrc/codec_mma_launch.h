@@ -1,0 +1,30 @@
+// Host-side entry to the tensor-core codec kernels.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include "ssn_common.cuh"
+
+namespace ssn {
+
+struct MmaArgs {
+  const __nv_bfloat16 *src;   // [n x d] rows to project, or nullptr (expand only)
+  const __nv_bfloat16 *zin;   // [n x k] coordinates for expand-only
+  __nv_bfloat16 *zout;        // [n x k] coordinates out, nullable
+  __nv_bfloat16 *dst;         // [n x d] expansion out, nullable
+  const __nv_bfloat16 *U;     // [d x k], 16-byte aligned, ldu % 8 == 0
+  int64_t lds, ldzin, ldzout, lddst, ldu;
+  int64_t n;
+  int32_t d, k;
+  ShiftTables shift;
+};
+
+// Shapes the tensor-core kernels take (alignment is checked by the caller).
+bool codec_mma_supports(int d, int k);
+
+// mode: 1 = project, 2 = expand, 3 = project then expand (shift must be false).
+cudaError_t launch_codec_mma(const MmaArgs &a, bool shift, int mode, int sm_count,
+                             cudaStream_t stream);
+
+}  // namespace ssn

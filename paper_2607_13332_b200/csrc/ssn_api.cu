@@ -7,6 +7,7 @@
 
 #include <atomic>
 
+#include "codec_mma_launch.h"
 #include "generic_kernels.cuh"
 #include "ssn_common.cuh"
 
@@ -56,8 +57,61 @@ ssn_status_t launch_status(int launches = 1) {
   return cudaGetLastError() == cudaSuccess ? SSN_OK : SSN_ERR_CUDA;
 }
 
+inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+int sm_count_of_current_device() {
+  static int cached[64];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
+  if (cached[dev] == 0) {
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) n = 0;
+    cached[dev] = n;
+  }
+  return cached[dev];
+}
+
+// True when the call can run on the tensor-core kernels: bf16, supported shape, every big
+// matrix 16-byte aligned with a leading dimension that keeps its rows 16-byte aligned.
+bool mma_eligible(const TokenArgs &a, int32_t dtype) {
+  if (dtype != SSN_BF16 || !codec_mma_supports(a.d, a.k)) return false;
+  if (!aligned16(a.U) || (a.ldu & 7)) return false;
+  if (a.src && (!aligned16(a.src) || (a.lds & 7))) return false;
+  if (a.dst && (!aligned16(a.dst) || (a.lddst & 7))) return false;
+  if (a.sub_shift || a.add_shift) {
+    if (a.shift.E && (!aligned16(a.shift.E) || (a.shift.lde & 7))) return false;
+    if (a.shift.P && (!aligned16(a.shift.P) || (a.shift.ldp & 7))) return false;
+  }
+  return true;
+}
+
 ssn_status_t launch_token_kernel(const TokenArgs &a, int32_t dtype, cudaStream_t stream) {
   if (a.n == 0) return SSN_OK;
+  if (mma_eligible(a, dtype)) {
+    const int sms = sm_count_of_current_device();
+    if (sms > 0) {
+      MmaArgs m{};
+      m.src = static_cast<const __nv_bfloat16 *>(a.src);
+      m.zin = static_cast<const __nv_bfloat16 *>(a.zin);
+      m.zout = static_cast<__nv_bfloat16 *>(a.zout);
+      m.dst = static_cast<__nv_bfloat16 *>(a.dst);
+      m.U = static_cast<const __nv_bfloat16 *>(a.U);
+      m.lds = a.lds;
+      m.ldzin = a.ldzin;
+      m.ldzout = a.ldzout;
+      m.lddst = a.lddst;
+      m.ldu = a.ldu;
+      m.n = a.n;
+      m.d = a.d;
+      m.k = a.k;
+      m.shift = a.shift;
+      const bool shift = (a.sub_shift || a.add_shift) && (a.shift.E || a.shift.P);
+      const int mode = (a.src ? 1 : 0) | (a.dst ? 2 : 0);
+      cudaError_t e = launch_codec_mma(m, shift, mode, sms, stream);
+      g_launches.fetch_add(1, std::memory_order_relaxed);
+      return e == cudaSuccess ? SSN_OK : SSN_ERR_CUDA;
+    }
+  }
   const int64_t blocks = (a.n + kGenericWarps - 1) / kGenericWarps;
   if (blocks > 0x7fffffffLL) return SSN_ERR_SHAPE;
   const size_t smem = (size_t)kGenericWarps * a.k * sizeof(float);
