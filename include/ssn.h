@@ -68,6 +68,7 @@ typedef enum { SSN_GRAD_COEFF = 1, SSN_GRAD_FULL = 2 } ssn_grad_mode_t;
 /* Bits of the device status word. */
 #define SSN_DEV_BAD_ID 1
 #define SSN_DEV_BAD_POS 2
+#define SSN_DEV_TIMEOUT 4   /* an internal bounded wait ran out; the output is invalid */
 
 /*
  * The data both ends of a stage boundary share (Sec. 4.1: the basis U_k, and PE and T_fixed

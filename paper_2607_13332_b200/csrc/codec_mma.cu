@@ -1,6 +1,7 @@
 // Instantiations and launcher of the tensor-core codec kernels (see codec_mma.cuh).
 #include "codec_mma.cuh"
 
+
 #include "codec_mma_launch.h"
 
 namespace ssn {
@@ -42,12 +43,23 @@ bool codec_mma_supports(int d, int k) {
 cudaError_t launch_codec_mma(const MmaArgs &a, bool shift, int mode, int sm_count,
                              cudaStream_t stream) {
   const int nt = (a.k + 7) / 8;
-  if (nt <= 1) return launch_nt<1, 2>(a, shift, mode, sm_count, stream);
-  if (nt <= 2) return launch_nt<2, 2>(a, shift, mode, sm_count, stream);
-  if (nt <= 4) return launch_nt<4, 2>(a, shift, mode, sm_count, stream);
-  if (nt <= 5) return launch_nt<5, 2>(a, shift, mode, sm_count, stream);
-  if (nt <= 6) return launch_nt<6, 2>(a, shift, mode, sm_count, stream);
-  if (nt <= 8) return launch_nt<8, 2>(a, shift, mode, sm_count, stream);
+  // With few tokens per warp a second 16-row tile would be computed for nothing.
+  const bool small = a.n <= (int64_t)sm_count * kMmaWarps * 16;
+  if (small) {
+    if (nt <= 1) return launch_nt<1, 1>(a, shift, mode, sm_count, stream);
+    if (nt <= 2) return launch_nt<2, 1>(a, shift, mode, sm_count, stream);
+    if (nt <= 4) return launch_nt<4, 1>(a, shift, mode, sm_count, stream);
+    if (nt <= 5) return launch_nt<5, 1>(a, shift, mode, sm_count, stream);
+    if (nt <= 6) return launch_nt<6, 1>(a, shift, mode, sm_count, stream);
+    if (nt <= 8) return launch_nt<8, 1>(a, shift, mode, sm_count, stream);
+  } else {
+    if (nt <= 1) return launch_nt<1, 2>(a, shift, mode, sm_count, stream);
+    if (nt <= 2) return launch_nt<2, 2>(a, shift, mode, sm_count, stream);
+    if (nt <= 4) return launch_nt<4, 2>(a, shift, mode, sm_count, stream);
+    if (nt <= 5) return launch_nt<5, 2>(a, shift, mode, sm_count, stream);
+    if (nt <= 6) return launch_nt<6, 2>(a, shift, mode, sm_count, stream);
+    if (nt <= 8) return launch_nt<8, 2>(a, shift, mode, sm_count, stream);
+  }
   if (nt <= 12) return launch_nt<12, 1>(a, shift, mode, sm_count, stream);
   return launch_nt<16, 1>(a, shift, mode, sm_count, stream);
 }

@@ -78,13 +78,36 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t *>(&v);
 }
+// Packed pair of fp32 in one 64-bit register (sm_100a has two-wide fp32 add/sub).
+__device__ __forceinline__ unsigned long long f32x2_of(uint32_t w) {
+  unsigned long long r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(w << 16), "r"(w & 0xffff0000u));
+  return r;
+}
+__device__ __forceinline__ unsigned long long f32x2_make(float lo, float hi) {
+  unsigned long long r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ uint32_t f32x2_to_bf16x2(unsigned long long v) {
+  uint32_t lo, hi, o;
+  asm("mov.b64 {%0, %1}, %2;" : "=r"(lo), "=r"(hi) : "l"(v));
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(o) : "r"(hi), "r"(lo));
+  return o;
+}
 // (x - e) - p on a pair of packed bf16, in fp32, rounded once to bf16.
 __device__ __forceinline__ uint32_t sub3(uint32_t x, uint32_t e, uint32_t p) {
-  return pack_bf16((bf_lo(x) - bf_lo(e)) - bf_lo(p), (bf_hi(x) - bf_hi(e)) - bf_hi(p));
+  unsigned long long r;
+  asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(f32x2_of(x)), "l"(f32x2_of(e)));
+  asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(r), "l"(f32x2_of(p)));
+  return f32x2_to_bf16x2(r);
 }
 // (acc + e) + p, rounded once.
 __device__ __forceinline__ uint32_t add3(float a0, float a1, uint32_t e, uint32_t p) {
-  return pack_bf16((a0 + bf_lo(e)) + bf_lo(p), (a1 + bf_hi(e)) + bf_hi(p));
+  unsigned long long r;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(f32x2_make(a0, a1)), "l"(f32x2_of(e)));
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(r), "l"(f32x2_of(p)));
+  return f32x2_to_bf16x2(r);
 }
 
 // ---- the U stage ring ------------------------------------------------------------------------
@@ -99,6 +122,7 @@ struct UStageRing {
   int64_t ldu;
   int d, k, nstage, total_jobs;
   uint32_t smem_base;
+  bool named_barrier = false;   // the kMmaThreads users are only part of the CTA
 
   __device__ __forceinline__ void issue(int job) {
     if (job < total_jobs) {
@@ -118,7 +142,10 @@ struct UStageRing {
   // Makes stage `job` readable by every warp and refills the buffer freed by job-1.
   __device__ __forceinline__ uint32_t acquire(int job) {
     cp_async_wait<1>();
-    __syncthreads();
+    if (named_barrier)
+      asm volatile("bar.sync 1, %0;\n" ::"n"(kMmaThreads) : "memory");
+    else
+      __syncthreads();
     issue(job + 2);
     return smem_base + (uint32_t)(job % kStages) * kStageBytes;
   }
@@ -201,60 +228,75 @@ __global__ void __launch_bounds__(kMmaThreads, 1) codec_mma_kernel(const MmaArgs
 
     // ------------------------------------------------------------------ projection pass
     if (has_project) {
+      // A ring of register buffers, one 32-column chunk each.  A buffer is refilled (chunk
+      // c + kPBuf) as soon as its contents have been turned into A fragments, before the MMAs
+      // of chunk c are issued, so close to kPBuf chunks of loads are in flight per thread.
       constexpr int NB = SHIFT ? 3 : 1;
-      uint4 bufA[MT][2][NB], bufB[MT][2][NB];
-      auto load = [&](uint4 (&buf)[MT][2][NB], int chunk) {
-        const int off = min(chunk, nchunks - 1) * 64;
+      constexpr int kPBuf = SHIFT ? 2 : 4;
+      uint4 buf[kPBuf][MT][2][NB];
+      auto load = [&](uint4 (&b)[MT][2][NB], int off) {
 #pragma unroll
         for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
           for (int h = 0; h < 2; ++h) {
-            buf[mt][h][0] = ldg16(xrow[mt][h] + off);
+            b[mt][h][0] = ldg16(xrow[mt][h] + off);
             if (SHIFT) {
-              buf[mt][h][1] = ldg16(erow[mt][h] + off);
-              buf[mt][h][2] = ldg16(prow[mt][h] + off);
+              b[mt][h][1] = ldg16(erow[mt][h] + off);
+              b[mt][h][2] = ldg16(prow[mt][h] + off);
             }
           }
       };
-      auto compute = [&](uint4 (&buf)[MT][2][NB], uint32_t ubase, int blk) {
-        uint32_t ra[MT][2][4];
+      auto convert = [&](uint4 (&b)[MT][2][NB], uint32_t (&ra)[MT][2][4]) {
 #pragma unroll
         for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
           for (int h = 0; h < 2; ++h) {
             if (SHIFT) {
-              ra[mt][h][0] = sub3(buf[mt][h][0].x, buf[mt][h][1].x, buf[mt][h][2].x);
-              ra[mt][h][1] = sub3(buf[mt][h][0].y, buf[mt][h][1].y, buf[mt][h][2].y);
-              ra[mt][h][2] = sub3(buf[mt][h][0].z, buf[mt][h][1].z, buf[mt][h][2].z);
-              ra[mt][h][3] = sub3(buf[mt][h][0].w, buf[mt][h][1].w, buf[mt][h][2].w);
+              ra[mt][h][0] = sub3(b[mt][h][0].x, b[mt][h][1].x, b[mt][h][2].x);
+              ra[mt][h][1] = sub3(b[mt][h][0].y, b[mt][h][1].y, b[mt][h][2].y);
+              ra[mt][h][2] = sub3(b[mt][h][0].z, b[mt][h][1].z, b[mt][h][2].z);
+              ra[mt][h][3] = sub3(b[mt][h][0].w, b[mt][h][1].w, b[mt][h][2].w);
             } else {
-              ra[mt][h][0] = buf[mt][h][0].x;
-              ra[mt][h][1] = buf[mt][h][0].y;
-              ra[mt][h][2] = buf[mt][h][0].z;
-              ra[mt][h][3] = buf[mt][h][0].w;
+              ra[mt][h][0] = b[mt][h][0].x;
+              ra[mt][h][1] = b[mt][h][0].y;
+              ra[mt][h][2] = b[mt][h][0].z;
+              ra[mt][h][3] = b[mt][h][0].w;
             }
           }
+      };
+      auto mmas = [&](uint32_t (&ra)[MT][2][4], uint32_t ubase, int blk) {
         const uint32_t bbase = ubase + (uint32_t)blk * (NT * 512) + lane_piece;
+        uint32_t b[NT][4];
 #pragma unroll
-        for (int nt = 0; nt < NT; ++nt) {
-          uint32_t b[4];
-          ldmatrix_x4_trans(b, bbase + nt * 512);
+        for (int nt = 0; nt < NT; ++nt) ldmatrix_x4_trans(b[nt], bbase + nt * 512);
+        // the two MMAs that share an accumulator are issued NT*MT instructions apart
 #pragma unroll
-          for (int mt = 0; mt < MT; ++mt) {
-            mma_k16(acc[mt][nt], ra[mt][0][0], ra[mt][1][0], ra[mt][0][1], ra[mt][1][1], b[0], b[1]);
-            mma_k16(acc[mt][nt], ra[mt][0][2], ra[mt][1][2], ra[mt][0][3], ra[mt][1][3], b[2], b[3]);
-          }
-        }
+        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+          for (int mt = 0; mt < MT; ++mt)
+            mma_k16(acc[mt][nt], ra[mt][0][0], ra[mt][1][0], ra[mt][0][1], ra[mt][1][1], b[nt][0], b[nt][1]);
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+          for (int mt = 0; mt < MT; ++mt)
+            mma_k16(acc[mt][nt], ra[mt][0][2], ra[mt][1][2], ra[mt][0][3], ra[mt][1][3], b[nt][2], b[nt][3]);
       };
 
-      load(bufA, 0);
-      uint32_t ubase = 0;
-      for (int c = 0; c < nchunks; c += 2) {
-        if ((c & 3) == 0) ubase = ring.acquire(job++);
-        load(bufB, c + 1);
-        compute(bufA, ubase, c & 3);
-        load(bufA, c + 2);
-        if (c + 1 < nchunks) compute(bufB, ubase, (c + 1) & 3);
+#pragma unroll
+      for (int i = 0; i < kPBuf; ++i)
+        if (i < nchunks) load(buf[i], i * 64);
+      for (int c0 = 0; c0 < nchunks; c0 += 4) {
+        const uint32_t ubase = ring.acquire(job++);
+        const int base_off = c0 * 64;
+#pragma unroll
+        for (int cc = 0; cc < 4; ++cc) {
+          if (c0 + cc < nchunks) {
+            uint32_t ra[MT][2][4];
+            convert(buf[cc % kPBuf], ra);
+            if (c0 + cc + kPBuf < nchunks) load(buf[cc % kPBuf], base_off + (cc + kPBuf) * 64);
+            mmas(ra, ubase, cc);
+          }
+        }
       }
 
       if (a.zout != nullptr) {
