@@ -1,5 +1,6 @@
 // Instantiations and launcher of the tensor-core codec kernels (see codec_mma.cuh).
 #include "codec_mma.cuh"
+#include "codec_umma.cuh"
 
 
 #include "codec_mma_launch.h"
@@ -34,7 +35,95 @@ cudaError_t launch_nt(const MmaArgs &a, bool shift, int mode, int sm_count, cuda
   return launch_one<NT, MT, false, kModeBoth>(a, sm_count, s);
 }
 
+// ---- tcgen05 / TMA projection ---------------------------------------------------------------
+using EncodeTiledFn = CUresult (*)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *,
+                                   const cuuint64_t *, const cuuint64_t *, const cuuint32_t *,
+                                   const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static bool tried = false;
+  if (!tried) {
+    tried = true;
+    void *p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+    else
+      cudaGetLastError();
+  }
+  return fn;
+}
+
+// Row-major bf16 matrix [rows x cols], leading dimension ld, fetched in boxes of box_rows x 64
+// columns into the 128-byte swizzled layout.
+bool make_sw128_map(CUtensorMap *map, const void *base, int64_t rows, int64_t cols, int64_t ld,
+                    int box_rows) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (fn == nullptr || rows < 1 || rows > 0x7fffffffLL) return false;
+  cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+  cuuint32_t box[2] = {(cuuint32_t)kUmmaCols, (cuuint32_t)box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box,
+            estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int NTP, bool HAS_E, bool HAS_P>
+cudaError_t launch_umma_one(const MmaArgs &a, const UmmaMaps &maps, int sm_count, cudaStream_t stream) {
+  auto kernel = codec_umma_project_kernel<NTP, HAS_E, HAS_P>;
+  constexpr int smem = UmmaProjectConfig<NTP, HAS_E, HAS_P>::kSmemBytes;
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  int64_t grid = (a.n + kUmmaTile - 1) / kUmmaTile;
+  if (grid > sm_count) grid = sm_count;
+  kernel<<<(unsigned)grid, kUmmaThreads, smem, stream>>>(a, maps);
+  return cudaGetLastError();
+}
+
+template <int NTP>
+cudaError_t launch_umma_ntp(const MmaArgs &a, bool has_e, bool has_p, const UmmaMaps &maps, int sm_count,
+                            cudaStream_t s) {
+  if (has_e && has_p) return launch_umma_one<NTP, true, true>(a, maps, sm_count, s);
+  if (has_e) return launch_umma_one<NTP, true, false>(a, maps, sm_count, s);
+  if (has_p) return launch_umma_one<NTP, false, true>(a, maps, sm_count, s);
+  return launch_umma_one<NTP, false, false>(a, maps, sm_count, s);
+}
+
 }  // namespace
+
+// Projection on tcgen05.  Returns cudaErrorNotSupported when the call should take the mma.sync
+// kernel instead: small batches, k not a multiple of 8, d not a multiple of 64, explicit or
+// wrapping positions inside a 128-token tile, no tensor map.
+cudaError_t launch_codec_umma_project(const MmaArgs &a, bool shift, int sm_count, cudaStream_t stream) {
+  if (a.zout == nullptr || a.dst != nullptr || a.src == nullptr) return cudaErrorNotSupported;
+  if (a.d % kUmmaCols != 0 || a.k % 8 != 0 || a.k > 128 || a.n < 4 * kUmmaTile || a.n > 0x7fffffffLL)
+    return cudaErrorNotSupported;
+  const bool has_e = shift && a.shift.E != nullptr, has_p = shift && a.shift.P != nullptr;
+  if (has_p && (a.shift.pos != nullptr || a.shift.seq_len % kUmmaTile != 0 ||
+                a.shift.seq_len > a.shift.max_pos))
+    return cudaErrorNotSupported;
+  const int ntp = 2 * ((a.k + 15) / 16);
+  UmmaMaps maps;
+  if (!make_sw128_map(&maps.x, a.src, a.n, a.d, a.lds, kUmmaTile)) return cudaErrorNotSupported;
+  if (!make_sw128_map(&maps.u, a.U, a.d, a.k, a.ldu, kUmmaCols)) return cudaErrorNotSupported;
+  maps.p = maps.x;
+  if (has_p && !make_sw128_map(&maps.p, a.shift.P, a.shift.max_pos, a.d, a.shift.ldp, kUmmaTile))
+    return cudaErrorNotSupported;
+  if (ntp <= 2) return launch_umma_ntp<2>(a, has_e, has_p, maps, sm_count, stream);
+  if (ntp <= 4) return launch_umma_ntp<4>(a, has_e, has_p, maps, sm_count, stream);
+  if (ntp <= 6) return launch_umma_ntp<6>(a, has_e, has_p, maps, sm_count, stream);
+  if (ntp <= 8) return launch_umma_ntp<8>(a, has_e, has_p, maps, sm_count, stream);
+  if (ntp <= 12) return launch_umma_ntp<12>(a, has_e, has_p, maps, sm_count, stream);
+  return launch_umma_ntp<16>(a, has_e, has_p, maps, sm_count, stream);
+}
 
 bool codec_mma_supports(int d, int k) {
   return d % 32 == 0 && (int64_t)d * 2 <= kZeroRowBytes && k >= 1 && k <= 128;
@@ -42,6 +131,10 @@ bool codec_mma_supports(int d, int k) {
 
 cudaError_t launch_codec_mma(const MmaArgs &a, bool shift, int mode, int sm_count,
                              cudaStream_t stream) {
+  if (mode == kModeProject) {
+    cudaError_t e = launch_codec_umma_project(a, shift, sm_count, stream);
+    if (e != cudaErrorNotSupported) return e;
+  }
   const int nt = (a.k + 7) / 8;
   // With few tokens per warp a second 16-row tile would be computed for nothing.
   const bool small = a.n <= (int64_t)sm_count * kMmaWarps * 16;

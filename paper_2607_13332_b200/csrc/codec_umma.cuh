@@ -1,0 +1,357 @@
+// tcgen05 / TMA projection kernel of the SSN codec (bf16, sm_100a):
+//     Z = X U - E[ids] U - P[pos] U        compress (SHIFT) / grad-project coefficients (!SHIFT)
+//
+// The subtraction of Eq. (ssn_compress) is moved through the contraction: the three products
+// are accumulated into one fp32 accumulator in tensor memory, the E and P products with the
+// instruction descriptor's negate-A bit set.  bf16 x bf16 products are exact in fp32, so the
+// only rounding is fp32 accumulation, and no thread ever touches an element of X, E or P:
+//
+//   warp 0   producer.  Per stage (128 tokens x 64 columns) one TMA box load of X, one of the
+//            P rows (positions of a tile are consecutive) and one of the 64 x k slice of U.
+//   warp 1   one thread issues tcgen05.mma (M=128, N=k rounded up to 16, K=16) for the stage and
+//            commits to the stage's "empty" barrier; the last stage of a tile also commits to the
+//            accumulator's "full" barrier.  This warp owns the TMEM allocation.
+//   warps 2-5  gather the E rows of the tile: 8 lanes copy one 128-byte row piece with cp.async
+//            straight into the swizzled tile, three stages ahead of the barrier arrival that
+//            publishes them (an id outside the table points at a row of zeros).
+//   warps 6-9  epilogue: tcgen05.ld their 32 TMEM lanes (one token per thread), round to bf16,
+//            store the Z rows; two accumulators let a tile's epilogue overlap the next tile's MMAs.
+//
+// X, E and P tiles use the 128-byte swizzled K-major layout (rows of 128 bytes); U arrives as a
+// 128-byte swizzled MN-major operand straight from its row-major storage.  Every wait is
+// bounded; a wait that runs out sets SSN_DEV_TIMEOUT and the kernel still runs to its end.
+#pragma once
+
+#include <cuda.h>
+
+#include "codec_mma.cuh"
+
+namespace ssn {
+
+constexpr int kUmmaThreads = 320;
+constexpr int kUmmaTile = 128;     // tokens per tile (MMA M)
+constexpr int kUmmaCols = 64;      // columns of X per stage (one 128-byte swizzle row)
+constexpr int kWaitSpins = 1 << 22;
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, int count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];\n" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n.reg .pred p;\n"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+      "selp.u32 %0, 1, 0, p;\n}\n"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Waits for the phase with the given parity; gives up (returns false) after kWaitSpins polls.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+  int spins = 0;
+  while (!mbar_try_wait(bar, parity))
+    if (++spins > kWaitSpins) return false;
+  return true;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, uint32_t bar,
+                                            int c0, int c1) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cta.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];\n"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1) : "memory");
+}
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *map, uint32_t bar,
+                                            int c0, int c1, int c2, int c3) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cta.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];\n"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+}
+__device__ __forceinline__ void tma_gather4(uint32_t dst, const CUtensorMap *map, uint32_t bar,
+                                            int c0, int r0, int r1, int r2, int r3) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cta.global.tile::gather4.mbarrier::complete_tx::bytes "
+      "[%0], [%1, {%3, %4, %5, %6, %7}], [%2];\n"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(r0), "r"(r1), "r"(r2), "r"(r3) : "memory");
+}
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc,
+                                          uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n.reg .pred p;\n"
+      "setp.ne.b32 p, %4, 0;\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];\n"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr));
+}
+
+// Shared-memory operand descriptors (64-bit): start address, leading / stride byte offsets in
+// 16-byte units, descriptor version 1, layout type in bits 61..63.
+__device__ __forceinline__ uint64_t umma_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes,
+                                              uint32_t layout_type) {
+  return (uint64_t)((addr >> 4) & 0x3FFFu) | ((uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16) |
+         ((uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32) | (1ull << 46) | ((uint64_t)layout_type << 61);
+}
+
+// Instruction descriptor: fp32 accumulate, bf16 A (K-major, optionally negated) and bf16 B
+// (MN-major), N and M encoded as N/8 and M/16.
+__host__ __device__ constexpr uint32_t umma_idesc(int n, bool negate_a) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((negate_a ? 1u : 0u) << 13) | (1u << 16) |
+         ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kUmmaTile >> 4) << 24);
+}
+
+template <int NTP, bool HAS_E, bool HAS_P>
+struct UmmaProjectConfig {
+  static_assert(NTP % 2 == 0 && NTP >= 2 && NTP <= 16, "N = 8*NTP must be a multiple of 16 up to 128");
+  static constexpr int kN = NTP * 8;
+  static constexpr int kATileBytes = kUmmaTile * 128;               // 128 rows of 128 bytes
+  static constexpr int kATiles = 1 + (HAS_E ? 1 : 0) + (HAS_P ? 1 : 0);
+  static constexpr int kUGroups = kN <= 64 ? 1 : 2;                 // 64-column groups of U
+  static constexpr int kUGroupBytes = kUmmaCols * 128;              // 64 rows of 128 bytes
+  static constexpr int kUBytes = kUGroups * kUGroupBytes;
+  static constexpr int kStageBytes = kATiles * kATileBytes + kUBytes;
+  static constexpr int kTmaBytes = kStageBytes - (HAS_E ? kATileBytes : 0);
+  static constexpr int kMaxSmem = 227 * 1024;
+  static constexpr int kFit = (kMaxSmem - 1024 - 512) / kStageBytes;
+  static constexpr int kStagesN = kFit < 8 ? kFit : 8;
+  static_assert(kStagesN >= 2, "no room for two stages");
+  static constexpr int kGatherLag = kStagesN > 3 ? 3 : kStagesN - 1;   // stages between issuing a gather and publishing it
+  static constexpr int kAccCols = kN <= 32 ? 32 : (kN <= 64 ? 64 : 128);   // TMEM columns per accumulator
+  static constexpr int kBarBytes = (2 * kStagesN + 4) * 8 + 16;
+  static constexpr int kSmemBytes = 1024 + kStagesN * kStageBytes + kBarBytes;
+};
+
+struct UmmaMaps {
+  CUtensorMap x, p, u;
+};
+
+template <int NTP, bool HAS_E, bool HAS_P>
+__global__ void __launch_bounds__(kUmmaThreads, 1)
+codec_umma_project_kernel(const MmaArgs a, const __grid_constant__ UmmaMaps maps) {
+  using Cfg = UmmaProjectConfig<NTP, HAS_E, HAS_P>;
+  constexpr int kETile = 1, kPTile = HAS_E ? 2 : 1;   // order of the tiles inside a stage
+  constexpr int S = Cfg::kStagesN;
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int nstage = a.d / kUmmaCols;
+  const int64_t ntiles = (a.n + kUmmaTile - 1) / kUmmaTile;
+
+  const uint32_t smem0 = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t bars = smem0 + S * Cfg::kStageBytes;
+  auto full_bar = [&](int s) { return bars + s * 8; };
+  auto empty_bar = [&](int s) { return bars + (S + s) * 8; };
+  auto acc_full_bar = [&](int b) { return bars + (2 * S + b) * 8; };
+  auto acc_empty_bar = [&](int b) { return bars + (2 * S + 2 + b) * 8; };
+  const uint32_t tmem_slot = bars + (2 * S + 4) * 8;
+  volatile uint32_t *tmem_slot_ptr =
+      reinterpret_cast<volatile uint32_t *>(smem_raw + (tmem_slot - smem_u32(smem_raw)));
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < S; ++s) {
+      mbar_init(full_bar(s), HAS_E ? 5 : 1);
+      mbar_init(empty_bar(s), 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(acc_full_bar(b), 1);
+      mbar_init(acc_empty_bar(b), 4);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(tmem_slot),
+                 "r"(2 * Cfg::kAccCols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+  const uint32_t tmem_base = *tmem_slot_ptr;
+  bool dead = false;
+  auto timed_out = [&]() {
+    dead = true;
+    if (a.shift.dev_status) atomicOr(a.shift.dev_status, SSN_DEV_TIMEOUT);
+  };
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------------- producer
+    int slot = 0;
+    uint32_t parity = 1;   // a fresh "empty" barrier passes a wait on parity 1
+    for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+      const int64_t tok0 = tile * kUmmaTile;
+      const int pos0 = HAS_P ? (int)(tok0 % a.shift.seq_len) : 0;
+      for (int st = 0; st < nstage; ++st) {
+        if (!dead && !mbar_wait(empty_bar(slot), parity)) timed_out();
+        const uint32_t base = smem0 + (uint32_t)slot * Cfg::kStageBytes;
+        const uint32_t bar = full_bar(slot);
+        if (lane == 0) {
+          mbar_expect_tx(bar, Cfg::kTmaBytes);
+          tma_load_2d(base, &maps.x, bar, st * kUmmaCols, (int)tok0);
+          if (HAS_P) tma_load_2d(base + kPTile * Cfg::kATileBytes, &maps.p, bar, st * kUmmaCols, pos0);
+#pragma unroll
+          for (int ug = 0; ug < Cfg::kUGroups; ++ug)
+            tma_load_2d(base + Cfg::kATiles * Cfg::kATileBytes + ug * Cfg::kUGroupBytes, &maps.u, bar, ug * 64,
+                        st * kUmmaCols);
+        }
+        __syncwarp();
+        if (++slot == S) {
+          slot = 0;
+          parity ^= 1u;
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------------- MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc_pos = umma_idesc(Cfg::kN, false), idesc_neg = umma_idesc(Cfg::kN, true);
+      int slot = 0;
+      uint32_t parity = 0;
+      int64_t tcount = 0;
+      for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x, ++tcount) {
+        const int buf = (int)(tcount & 1);
+        const uint32_t acc_parity = (uint32_t)((tcount >> 1) & 1);
+        if (!dead && !mbar_wait(acc_empty_bar(buf), acc_parity ^ 1u)) timed_out();
+        asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+        const uint32_t d_tmem = tmem_base + (uint32_t)buf * Cfg::kAccCols;
+        for (int st = 0; st < nstage; ++st) {
+          if (!dead && !mbar_wait(full_bar(slot), parity)) timed_out();
+          asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+          const uint32_t base = smem0 + (uint32_t)slot * Cfg::kStageBytes;
+          const uint32_t ubase = base + Cfg::kATiles * Cfg::kATileBytes;
+#pragma unroll
+          for (int j = 0; j < kUmmaCols / 16; ++j) {
+            // U slice: rows are the contracted index (16 rows = 2048 bytes per K step), 64-column
+            // groups kUGroupBytes apart, 8-row groups 1024 bytes apart
+            const uint64_t bdesc = umma_desc(ubase + j * 2048, Cfg::kUGroupBytes, 1024, 2);
+            const uint64_t xdesc = umma_desc(base + j * 32, 16, 1024, 2);
+            umma_bf16(d_tmem, xdesc, bdesc, idesc_pos, (st > 0 || j > 0) ? 1u : 0u);
+            if (HAS_E) {
+              const uint64_t edesc = umma_desc(base + kETile * Cfg::kATileBytes + j * 32, 16, 1024, 2);
+              umma_bf16(d_tmem, edesc, bdesc, idesc_neg, 1u);
+            }
+            if (HAS_P) {
+              const uint64_t pdesc = umma_desc(base + kPTile * Cfg::kATileBytes + j * 32, 16, 1024, 2);
+              umma_bf16(d_tmem, pdesc, bdesc, idesc_neg, 1u);
+            }
+          }
+          umma_commit(empty_bar(slot));
+          if (st == nstage - 1) umma_commit(acc_full_bar(buf));
+          if (++slot == S) {
+            slot = 0;
+            parity ^= 1u;
+          }
+        }
+      }
+    }
+  } else if (warp < 6) {
+    // ------------------------------------------------------------------------- E row gather
+    if (HAS_E) {
+      const int gw = warp - 2;                 // rows 32*gw .. 32*gw+31 of the tile
+      const int piece = lane & 7, sub = lane >> 3;
+      int slot = 0, pub_slot = 0, pending = 0;
+      uint32_t parity = 1;
+      auto publish = [&]() {                   // the oldest issued stage has landed
+        asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
+        __syncwarp();
+        if (lane == 0) mbar_arrive(full_bar(pub_slot));
+        if (++pub_slot == S) pub_slot = 0;
+        --pending;
+      };
+      for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+        const int64_t tok0 = tile * kUmmaTile;
+        const unsigned char *src[8];
+        uint32_t dst[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const int r = gw * 32 + i * 4 + sub;
+          const int64_t t = tok0 + r;
+          const int64_t er = t < a.n ? embedding_row(a.shift, t) : -1;
+          src[i] = (er >= 0 ? reinterpret_cast<const unsigned char *>(
+                                  static_cast<const __nv_bfloat16 *>(a.shift.E) + er * a.shift.lde)
+                            : g_zero_row) + piece * 16;
+          dst[i] = kETile * Cfg::kATileBytes + r * 128 + ((piece ^ (r & 7)) << 4);
+        }
+        for (int st = 0; st < nstage; ++st) {
+          if (!dead && !mbar_wait(empty_bar(slot), parity)) timed_out();
+          const uint32_t base = smem0 + (uint32_t)slot * Cfg::kStageBytes;
+#pragma unroll
+          for (int i = 0; i < 8; ++i) cp_async16(base + dst[i], src[i] + st * 128, 16);
+          cp_async_commit();
+          if (++pending > Cfg::kGatherLag) {
+            cp_async_wait<Cfg::kGatherLag>();
+            publish();
+          }
+          if (++slot == S) {
+            slot = 0;
+            parity ^= 1u;
+          }
+        }
+      }
+      cp_async_wait<0>();
+      while (pending > 0) publish();
+    }
+  } else {
+    // ------------------------------------------------------------------------- epilogue
+    const int quarter = warp & 3;   // the TMEM lanes this warp may read: 32*quarter .. +31
+    int64_t tcount = 0;
+    const bool vec = ((a.ldzout & 7) == 0) && ((reinterpret_cast<uintptr_t>(a.zout) & 15) == 0);
+    for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x, ++tcount) {
+      const int buf = (int)(tcount & 1);
+      const uint32_t acc_parity = (uint32_t)((tcount >> 1) & 1);
+      if (!dead && !mbar_wait(acc_full_bar(buf), acc_parity)) timed_out();
+      asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+      const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)buf * Cfg::kAccCols;
+      uint32_t v[Cfg::kN / 16][16];
+#pragma unroll
+      for (int q = 0; q < Cfg::kN / 16; ++q) tmem_ld16(taddr + q * 16, v[q]);
+      asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
+      asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
+      __syncwarp();
+      if (lane == 0) mbar_arrive(acc_empty_bar(buf));
+
+      const int64_t t = tile * kUmmaTile + quarter * 32 + lane;
+      if (t < a.n) {
+        __nv_bfloat16 *zrow = a.zout + t * a.ldzout;
+#pragma unroll
+        for (int q = 0; q < Cfg::kN / 16; ++q) {
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            const int col = q * 16 + h * 8;
+            if (vec && col + 8 <= a.k) {
+              uint4 o;
+              o.x = pack_bf16(__uint_as_float(v[q][h * 8 + 0]), __uint_as_float(v[q][h * 8 + 1]));
+              o.y = pack_bf16(__uint_as_float(v[q][h * 8 + 2]), __uint_as_float(v[q][h * 8 + 3]));
+              o.z = pack_bf16(__uint_as_float(v[q][h * 8 + 4]), __uint_as_float(v[q][h * 8 + 5]));
+              o.w = pack_bf16(__uint_as_float(v[q][h * 8 + 6]), __uint_as_float(v[q][h * 8 + 7]));
+              *reinterpret_cast<uint4 *>(zrow + col) = o;
+            } else {
+#pragma unroll
+              for (int i = 0; i < 8; ++i)
+                if (col + i < a.k) zrow[col + i] = __float2bfloat16_rn(__uint_as_float(v[q][h * 8 + i]));
+            }
+          }
+        }
+      }
+    }
+  }
+
+  asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
+  __syncthreads();
+  if (warp == 1) {
+    asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem_base),
+                 "r"(2 * Cfg::kAccCols) : "memory");
+  }
+}
+
+}  // namespace ssn
