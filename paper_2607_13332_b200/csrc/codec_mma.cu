@@ -100,11 +100,11 @@ cudaError_t launch_umma_ntp(const MmaArgs &a, bool has_e, bool has_p, const Umma
 }  // namespace
 
 // Projection on tcgen05.  Returns cudaErrorNotSupported when the call should take the mma.sync
-// kernel instead: small batches, k not a multiple of 8, d not a multiple of 64, explicit or
+// kernel instead: small batches, k > 128, d not a multiple of 64, explicit or
 // wrapping positions inside a 128-token tile, no tensor map.
 cudaError_t launch_codec_umma_project(const MmaArgs &a, bool shift, int sm_count, cudaStream_t stream) {
   if (a.zout == nullptr || a.dst != nullptr || a.src == nullptr) return cudaErrorNotSupported;
-  if (a.d % kUmmaCols != 0 || a.k % 8 != 0 || a.k > 128 || a.n < 4 * kUmmaTile || a.n > 0x7fffffffLL)
+  if (a.d % kUmmaCols != 0 || a.k > 128 || a.n < 4 * kUmmaTile || a.n > 0x7fffffffLL)
     return cudaErrorNotSupported;
   const bool has_e = shift && a.shift.E != nullptr, has_p = shift && a.shift.P != nullptr;
   if (has_p && (a.shift.pos != nullptr || a.shift.seq_len % kUmmaTile != 0 ||

@@ -372,11 +372,13 @@ __global__ void __launch_bounds__(kMmaThreads, 1) codec_mma_kernel(const MmaArgs
         for (int h = 0; h < 2; ++h)
           orow[mt][h] = reinterpret_cast<unsigned char *>(a.dst + tok[mt][h] * a.lddst) + tg * 16;
 
+      // Register ring of kEBuf chunks of E/P pieces: the buffer of chunk c is refilled with
+      // chunk c + kEBuf right after it has been added to the accumulators.
       constexpr int NBE = SHIFT ? 2 : 1;
-      uint4 ebufA[MT][2][NBE], ebufB[MT][2][NBE];
-      auto eload = [&](uint4 (&buf)[MT][2][NBE], int chunk) {
+      constexpr int kEBuf = 4;
+      uint4 ebuf[kEBuf][MT][2][NBE];
+      auto eload = [&](uint4 (&buf)[MT][2][NBE], int off) {
         if (SHIFT) {
-          const int off = min(chunk, nchunks - 1) * 64;
 #pragma unroll
           for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
@@ -386,7 +388,7 @@ __global__ void __launch_bounds__(kMmaThreads, 1) codec_mma_kernel(const MmaArgs
             }
         }
       };
-      auto ecompute = [&](uint4 (&buf)[MT][2][NBE], uint32_t ubase, int blk, int chunk) {
+      auto ecompute = [&](uint4 (&buf)[MT][2][NBE], uint32_t ubase, int blk, int off, bool refill) {
         float o[MT][4][4];
 #pragma unroll
         for (int mt = 0; mt < MT; ++mt)
@@ -428,7 +430,6 @@ __global__ void __launch_bounds__(kMmaThreads, 1) codec_mma_kernel(const MmaArgs
                 for (int j = 0; j < 4; ++j) mma_k8(o[mt][j], za[p][mt][ks][0], za[p][mt][ks][1], b[j]);
           }
         }
-        const int off = chunk * 64;
 #pragma unroll
         for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
@@ -447,16 +448,19 @@ __global__ void __launch_bounds__(kMmaThreads, 1) codec_mma_kernel(const MmaArgs
             }
             if (own[mt][h]) *reinterpret_cast<uint4 *>(orow[mt][h] + off) = v;
           }
+        if (refill) eload(buf, off + kEBuf * 64);
       };
 
-      eload(ebufA, 0);
-      uint32_t ubase = 0;
-      for (int c = 0; c < nchunks; c += 2) {
-        if ((c & 3) == 0) ubase = ring.acquire(job++);
-        eload(ebufB, c + 1);
-        ecompute(ebufA, ubase, c & 3, c);
-        eload(ebufA, c + 2);
-        if (c + 1 < nchunks) ecompute(ebufB, ubase, (c + 1) & 3, c + 1);
+#pragma unroll
+      for (int i = 0; i < kEBuf; ++i)
+        if (i < nchunks) eload(ebuf[i], i * 64);
+      for (int c0 = 0; c0 < nchunks; c0 += 4) {
+        const uint32_t ubase = ring.acquire(job++);
+        const int base_off = c0 * 64;
+#pragma unroll
+        for (int cc = 0; cc < 4; ++cc)
+          if (c0 + cc < nchunks)
+            ecompute(ebuf[cc % kEBuf], ubase, cc, base_off + cc * 64, c0 + cc + kEBuf < nchunks);
       }
     }
   }
