@@ -1,5 +1,6 @@
 // Instantiations and launcher of the tensor-core codec kernels (see codec_mma.cuh).
 #include "codec_mma.cuh"
+#include "codec_mma_dsplit.cuh"
 #include "codec_umma.cuh"
 
 
@@ -33,6 +34,43 @@ cudaError_t launch_nt(const MmaArgs &a, bool shift, int mode, int sm_count, cuda
     return shift ? launch_one<NT, MT, true, kModeExpand>(a, sm_count, s)
                  : launch_one<NT, MT, false, kModeExpand>(a, sm_count, s);
   return launch_one<NT, MT, false, kModeBoth>(a, sm_count, s);
+}
+
+template <int NT, int MT, bool SHIFT, int MODE>
+cudaError_t launch_dsplit_one(const MmaArgs &a, int sm_count, cudaStream_t stream) {
+  auto kernel = codec_mma_dsplit_kernel<NT, MT, SHIFT, MODE>;
+  constexpr int smem = DsplitConfig<NT, MT>::kSmemBytes;
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  int64_t grid = (a.n + 16 * MT - 1) / (16 * MT);
+  if (grid > sm_count) grid = sm_count;
+  kernel<<<(unsigned)grid, kMmaThreads, smem, stream>>>(a);
+  return cudaGetLastError();
+}
+
+template <int NT, int MT>
+cudaError_t launch_dsplit_nt(const MmaArgs &a, bool shift, int mode, int sm_count, cudaStream_t s) {
+  if (mode == kModeProject)
+    return shift ? launch_dsplit_one<NT, MT, true, kModeProject>(a, sm_count, s)
+                 : launch_dsplit_one<NT, MT, false, kModeProject>(a, sm_count, s);
+  if (mode == kModeExpand)
+    return shift ? launch_dsplit_one<NT, MT, true, kModeExpand>(a, sm_count, s)
+                 : launch_dsplit_one<NT, MT, false, kModeExpand>(a, sm_count, s);
+  return launch_dsplit_one<NT, MT, false, kModeBoth>(a, sm_count, s);
+}
+
+template <int MT>
+cudaError_t launch_dsplit(const MmaArgs &a, bool shift, int mode, int nt, int sm_count, cudaStream_t s) {
+  if (nt <= 1) return launch_dsplit_nt<1, MT>(a, shift, mode, sm_count, s);
+  if (nt <= 2) return launch_dsplit_nt<2, MT>(a, shift, mode, sm_count, s);
+  if (nt <= 4) return launch_dsplit_nt<4, MT>(a, shift, mode, sm_count, s);
+  if (nt <= 5) return launch_dsplit_nt<5, MT>(a, shift, mode, sm_count, s);
+  if (nt <= 6) return launch_dsplit_nt<6, MT>(a, shift, mode, sm_count, s);
+  return launch_dsplit_nt<8, MT>(a, shift, mode, sm_count, s);
 }
 
 // ---- tcgen05 / TMA projection ---------------------------------------------------------------
@@ -138,6 +176,11 @@ cudaError_t launch_codec_mma(const MmaArgs &a, bool shift, int mode, int sm_coun
   const int nt = (a.k + 7) / 8;
   // With few tokens per warp a second 16-row tile would be computed for nothing.
   const bool small = a.n <= (int64_t)sm_count * kMmaWarps * 16;
+  if (small && nt <= 8) {
+    // few rows per SM: the warps of a CTA share a row tile and split d
+    return a.n > (int64_t)sm_count * 16 ? launch_dsplit<2>(a, shift, mode, nt, sm_count, stream)
+                                        : launch_dsplit<1>(a, shift, mode, nt, sm_count, stream);
+  }
   if (small) {
     if (nt <= 1) return launch_nt<1, 1>(a, shift, mode, sm_count, stream);
     if (nt <= 2) return launch_nt<2, 1>(a, shift, mode, sm_count, stream);

@@ -115,9 +115,9 @@ __device__ __forceinline__ uint32_t add3(float a0, float a1, uint32_t e, uint32_
 //   (((dl/32)*NT + c)*4 + ((dl/2)%4))*8 + ((dl/8)%4)*2 + dl%2
 // so that the four 8x8 tiles a warp fetches for one (32-row block, chunk) are 512 contiguous
 // bytes, both for the transposed loads of the projection and the plain loads of the expansion.
-template <int NT>
+template <int NT, int ROWS = kStageRows>
 struct UStageRing {
-  static constexpr int kStageBytes = kStageRows * NT * 16;
+  static constexpr int kStageBytes = ROWS * NT * 16;
   const __nv_bfloat16 *U;
   int64_t ldu;
   int d, k, nstage, total_jobs;
@@ -127,8 +127,8 @@ struct UStageRing {
   __device__ __forceinline__ void issue(int job) {
     if (job < total_jobs) {
       const int s = job % nstage;
-      const int row0 = s * kStageRows;
-      const int rows = min(kStageRows, d - row0);
+      const int row0 = s * ROWS;
+      const int rows = min(ROWS, d - row0);
       const uint32_t base = smem_base + (uint32_t)(job % kStages) * kStageBytes;
       for (int idx = threadIdx.x; idx < rows * NT; idx += kMmaThreads) {
         const int dl = idx / NT, c = idx - dl * NT;
