@@ -38,9 +38,13 @@ METRIC = "ssn_codec_tokens_per_s"
 UNIT = "tokens/s"
 FALLBACK_HBM_GBS = 6650.0
 
-# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of ONE launch of the dominant
-# kernel on this workload, from the ncu capture summarised under profiles/; None until captured.
-NCU_TRAFFIC_BYTES = {"compress": None}
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of ONE launch of each kernel on the
+# default workload, from the ncu captures summarised under profiles/; None where not captured.
+NCU_TRAFFIC_BYTES = {"compress": 765.1e6, "decompress": 652.9e6, "grad_project": 541.1e6,
+                     "weight_reproject": 210.1e6}
+
+
+REPROJECT_ROWS_COLS = ((4096, 4096), (14336, 4096))
 
 
 def parse_args():
@@ -87,6 +91,9 @@ def algorithmic_bytes(wl, ids, step):
         return n * d * b + shift + d * k * b + n * k * b
     if step == "grad_project":
         return n * d * b + d * k * b + n * k * b
+    if step == "weight_reproject":        # both weights of one block, read once and written once
+        rows = sum(r for r, _ in REPROJECT_ROWS_COLS)
+        return 2 * rows * d * b + 2 * d * k * b
     raise ValueError(step)
 
 
@@ -265,18 +272,24 @@ def run_ours(args):
     stream = torch.cuda.current_stream()
     kernel_events = []
 
-    def step(record=False):
-        if record:
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record(stream)
-        codec.compress(X, ids, seq_len=wl.seq_len, out=Z)
-        if record:
-            e1.record(stream)
-            kernel_events.append((e0, e1))
-        codec.decompress(Z, ids, seq_len=wl.seq_len, out=Xh)
-        codec.grad_project(G, out=dZ)
+    def reproject():
         for g, ws in zip(groups, work):
             codec.weight_reproject(g, "right", workspace=ws)
+
+    calls = (("compress", lambda: codec.compress(X, ids, seq_len=wl.seq_len, out=Z)),
+             ("decompress", lambda: codec.decompress(Z, ids, seq_len=wl.seq_len, out=Xh)),
+             ("grad_project", lambda: codec.grad_project(G, out=dZ)),
+             ("weight_reproject", reproject))
+
+    def step(record=False):
+        for name, call in calls:
+            if record:
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+            call()
+            if record:
+                e1.record(stream)
+                kernel_events.append((name, e0, e1))
 
     def e2e_step():
         X.copy_(X_h, non_blocking=True)
@@ -312,10 +325,11 @@ def run_ours(args):
     t_begin = time.perf_counter()
     ms_total = timed(step, args.steps)
     launches = binding.ssn_launch_count() - launches0
-    # same loop once more with events around the dominant kernel (events add small gaps, so
-    # this pass is not the one that gives `value`)
+    # same loop once more with events around every call (events add small gaps, so this pass
+    # is not the one that gives `value`)
     timed(step, args.steps, record=True)
-    compress_ms = float(np.mean([a.elapsed_time(b) for a, b in kernel_events]))
+    kernel_ms = {name: float(np.mean([a.elapsed_time(b) for n_, a, b in kernel_events if n_ == name]))
+                 for name, _ in calls}
     for _ in range(2):
         e2e_step()
     ms_e2e = timed(e2e_step, args.steps)
@@ -330,8 +344,15 @@ def run_ours(args):
         ms_per_step = ms_total / args.steps
         value = world * n / (ms_per_step * 1e-3)
         peak, peak_kind = measured_hbm_peak()
-        algo = algorithmic_bytes(wl, t["ids"], "compress")
-        achieved = algo / (compress_ms * 1e-3) / 1e9
+        kernels = {}
+        for name, ms in kernel_ms.items():
+            algo_k = algorithmic_bytes(wl, t["ids"], name)
+            gbs = algo_k / (ms * 1e-3) / 1e9
+            kernels[name] = {"ms": ms, "algorithmic_bytes": algo_k, "achieved": gbs, "frac": gbs / peak,
+                             "traffic": NCU_TRAFFIC_BYTES.get(name)}
+        # the roofline object describes the call that takes the largest share of the step
+        dominant = max(kernel_ms, key=kernel_ms.get)
+        algo, achieved = kernels[dominant]["algorithmic_bytes"], kernels[dominant]["achieved"]
         h2d = X_h.numel() * 2 + G_h.numel() * 2 + ids_h.numel() * 4
         d2h = Z_h.numel() * 2 + dZ_h.numel() * 2
         out = {
@@ -339,10 +360,11 @@ def run_ours(args):
             "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": config_of(wl, world),
-            "roofline": {"bound": "hbm", "kernel": "ssn_compress", "achieved": achieved,
+            "roofline": {"bound": "hbm", "kernel": "ssn_" + dominant, "achieved": achieved,
                          "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "peak_kind": peak_kind, "algorithmic_bytes": algo,
-                         "kernel_ms": compress_ms, "traffic": NCU_TRAFFIC_BYTES["compress"]},
+                         "kernel_ms": kernel_ms[dominant], "traffic": NCU_TRAFFIC_BYTES.get(dominant),
+                         "kernels": kernels},
             "e2e": {"value": world * n / (ms_e2e / args.steps * 1e-3), "unit": UNIT,
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
             "gpu_launches": int(launches),
