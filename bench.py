@@ -238,14 +238,12 @@ def run_ours(args):
 
     import __graft_entry__ as entry
     entry.build()
-    from paper_2607_13332_b200 import binding, synth
+    from paper_2607_13332_b200 import binding, dist_util, synth
     from paper_2607_13332_b200.runner import Codec, to_device
 
     if not torch.cuda.is_available():
         raise RuntimeError("bench.py needs a CUDA device: the SSN codec has no CPU path")
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    rank, world, local = dist_util.rank_world()
     torch.cuda.set_device(local)
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
@@ -301,8 +299,7 @@ def run_ours(args):
 
     def barrier():
         torch.cuda.synchronize()
-        if world > 1:
-            dist.barrier()
+        dist_util.barrier()
         torch.cuda.synchronize()
 
     def timed(fn, steps, **kw):
@@ -313,10 +310,7 @@ def run_ours(args):
             fn(**kw)
         b.record(stream)
         barrier()
-        ms = torch.tensor([a.elapsed_time(b)], device="cuda")
-        if world > 1:
-            dist.all_reduce(ms, op=dist.ReduceOp.MAX)
-        return float(ms.item())
+        return dist_util.max_over_ranks(a.elapsed_time(b), device="cuda")
 
     for _ in range(max(3, args.warmup)):
         step()
