@@ -147,6 +147,35 @@ ssn_status_t ssn_weight_reproject(const ssn_codec_t *codec, void *const *W_ptrs,
                                   int64_t rows, int64_t cols, int64_t ldw, int32_t side,
                                   void *workspace, size_t workspace_bytes, void *stream);
 
+/*
+ * LEFT re-projection of ONE weight, W [d x cols] <- U (U^T W), without a caller workspace.
+ * (The paper has no counterpart: this is a packaging variant of ssn_weight_reproject.)
+ *
+ * Who needs it: processes that gave all their device memory to an arena at start-up, or that
+ * sit inside a latency-critical loop, cannot call cudaMalloc (it may fail, and it synchronises
+ * the device) and may have no spare buffer to lend as workspace.  For them the k x cols fp32
+ * coordinates U^T W are kept in a fixed SSN_STATIC_SCRATCH_BYTES array inside the library
+ * (every GPU that loads the library holds it until the process exits).  The call allocates
+ * nothing, frees nothing and calls no allocating library routine.
+ *
+ *   W     device [d x cols], leading dimension ldw >= cols, updated in place.
+ *   Limit: k * cols * 4 bytes must not exceed ssn_static_scratch_bytes(); a larger problem is
+ *          refused with SSN_ERR_WORKSPACE before anything is launched (use ssn_weight_reproject
+ *          with your own workspace for those).
+ *   First call on a device: looks up the device address of the scratch array (the device must
+ *          be current, as for every call).  Make that first call outside any stream capture.
+ *   Sharing: every call on a device uses the same array.  Its contents are rewritten completely
+ *          by each call, so nothing has to be cleared, but two calls that overlap on the GPU
+ *          (different streams, no ordering between them) race on it: order them.
+ * Same arithmetic and results as ssn_weight_reproject(..., SSN_SIDE_LEFT, ...) on one weight.
+ */
+#define SSN_STATIC_SCRATCH_BYTES (4u << 20)
+ssn_status_t ssn_weight_reproject_left_static(const ssn_codec_t *codec, void *W, int64_t cols,
+                                              int64_t ldw, void *stream);
+
+/* Size of the fixed scratch array used by ssn_weight_reproject_left_static. */
+size_t ssn_static_scratch_bytes(void);
+
 /* Static, never-NULL description of a status code. */
 const char *ssn_status_string(ssn_status_t status);
 

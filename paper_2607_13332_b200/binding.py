@@ -63,6 +63,8 @@ _SIGNATURES = {
     "ssn_weight_reproject_workspace_bytes": (_sz, [_codec_p, _i64, _i64, _i32, _i32]),
     "ssn_weight_reproject": (_i32, [_codec_p, ctypes.POINTER(_vp), _i32, _i64, _i64, _i64, _i32,
                                     _vp, _sz, _vp]),
+    "ssn_weight_reproject_left_static": (_i32, [_codec_p, _vp, _i64, _i64, _vp]),
+    "ssn_static_scratch_bytes": (_sz, []),
     "ssn_status_string": (ctypes.c_char_p, [_i32]),
     "ssn_version": (_i32, []),
     "ssn_launch_count": (_i64, []),
@@ -143,6 +145,19 @@ def ssn_weight_reproject(codec: ssn_codec_t, W_ptrs: Sequence[int], rows: int, c
     _check(_lib.ssn_weight_reproject(ctypes.byref(codec), arr, len(W_ptrs), rows, cols, ldw, side,
                                      workspace or None, workspace_bytes, stream or None),
            "ssn_weight_reproject")
+
+
+def ssn_static_scratch_bytes() -> int:
+    return int(_lib.ssn_static_scratch_bytes())
+
+
+def ssn_weight_reproject_left_static(codec: ssn_codec_t, W: int, cols: int, ldw: int,
+                                     stream: int = 0) -> None:
+    """LEFT re-projection of one weight [d x cols] using the library's fixed scratch array: for
+    callers that cannot allocate or lend a workspace.  Raises SsnError(SSN_ERR_WORKSPACE) when
+    k * cols * 4 exceeds ssn_static_scratch_bytes()."""
+    _check(_lib.ssn_weight_reproject_left_static(ctypes.byref(codec), W or None, cols, ldw,
+                                                 stream or None), "ssn_weight_reproject_left_static")
 
 
 def raw(name: str):
