@@ -1,6 +1,7 @@
 // Instantiations and launcher of the tensor-core codec kernels (see codec_mma.cuh).
 #include "codec_mma.cuh"
 #include "codec_mma_dsplit.cuh"
+#include "codec_expand64.cuh"
 #include "codec_umma.cuh"
 
 
@@ -71,6 +72,49 @@ cudaError_t launch_dsplit(const MmaArgs &a, bool shift, int mode, int nt, int sm
   if (nt <= 5) return launch_dsplit_nt<5, MT>(a, shift, mode, sm_count, s);
   if (nt <= 6) return launch_dsplit_nt<6, MT>(a, shift, mode, sm_count, s);
   return launch_dsplit_nt<8, MT>(a, shift, mode, sm_count, s);
+}
+
+template <int NT, int MT, bool SHIFT, bool PDEDUP>
+cudaError_t launch_expand64_one(const MmaArgs &a, int sm_count, cudaStream_t stream) {
+  auto kernel = codec_expand64_kernel<NT, MT, SHIFT, PDEDUP>;
+  constexpr int smem = kStages * UStageRing64<NT>::kStageBytes;
+  static bool configured = false;
+  if (smem > 48 * 1024 && !configured) {
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  kernel<<<(unsigned)sm_count, kMmaThreads, smem, stream>>>(a);
+  return cudaGetLastError();
+}
+
+template <int NT>
+cudaError_t launch_expand64_nt(const MmaArgs &a, bool shift, bool dedup, int sm_count, cudaStream_t s) {
+  if (!shift) return launch_expand64_one<NT, 2, false, false>(a, sm_count, s);
+  if (dedup) return launch_expand64_one<NT, 2, true, true>(a, sm_count, s);
+  return launch_expand64_one<NT, 1, true, false>(a, sm_count, s);
+}
+
+inline bool aligned32(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 31) == 0; }
+
+// Expansion with 64-column chunks; cudaErrorNotSupported sends the call to the 32-column kernel.
+cudaError_t launch_expand64(const MmaArgs &a, bool shift, int sm_count, cudaStream_t stream) {
+  const int nt = (a.k + 7) / 8;
+  if (a.d % 64 != 0 || nt > 8 || !aligned32(a.dst) || (a.lddst & 15)) return cudaErrorNotSupported;
+  bool dedup = false;
+  if (shift) {
+    if (a.shift.E && (!aligned32(a.shift.E) || (a.shift.lde & 15))) return cudaErrorNotSupported;
+    if (a.shift.P && (!aligned32(a.shift.P) || (a.shift.ldp & 15))) return cudaErrorNotSupported;
+    // tiles of 16 batch entries at one position: implicit positions, whole sequences, batch % 16 == 0
+    dedup = a.shift.P != nullptr && a.shift.pos == nullptr && a.shift.seq_len >= 1 &&
+            a.n % a.shift.seq_len == 0 && (a.n / a.shift.seq_len) % 16 == 0;
+  }
+  if (nt <= 1) return launch_expand64_nt<1>(a, shift, dedup, sm_count, stream);
+  if (nt <= 2) return launch_expand64_nt<2>(a, shift, dedup, sm_count, stream);
+  if (nt <= 4) return launch_expand64_nt<4>(a, shift, dedup, sm_count, stream);
+  if (nt <= 5) return launch_expand64_nt<5>(a, shift, dedup, sm_count, stream);
+  if (nt <= 6) return launch_expand64_nt<6>(a, shift, dedup, sm_count, stream);
+  return launch_expand64_nt<8>(a, shift, dedup, sm_count, stream);
 }
 
 // ---- tcgen05 / TMA projection ---------------------------------------------------------------
@@ -180,6 +224,10 @@ cudaError_t launch_codec_mma(const MmaArgs &a, bool shift, int mode, int sm_coun
     // few rows per SM: the warps of a CTA share a row tile and split d
     return a.n > (int64_t)sm_count * 16 ? launch_dsplit<2>(a, shift, mode, nt, sm_count, stream)
                                         : launch_dsplit<1>(a, shift, mode, nt, sm_count, stream);
+  }
+  if (!small && mode == kModeExpand) {
+    cudaError_t e = launch_expand64(a, shift, sm_count, stream);
+    if (e != cudaErrorNotSupported) return e;
   }
   if (small) {
     if (nt <= 1) return launch_nt<1, 1>(a, shift, mode, sm_count, stream);

@@ -33,7 +33,7 @@ constexpr int kZeroRowBytes = 65536;
 
 // A row of zeros that stands in for the E / P row of a token that has none (absent table,
 // index out of range, row past the end of the batch).  Never written.
-__device__ __align__(16) unsigned char g_zero_row[kZeroRowBytes];
+__device__ __align__(128) unsigned char g_zero_row[kZeroRowBytes];
 
 
 // ---- small PTX wrappers --------------------------------------------------------------------
