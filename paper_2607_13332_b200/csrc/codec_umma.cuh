@@ -8,9 +8,11 @@
 //
 //   warp 0   producer.  Per stage (128 tokens x 64 columns) one TMA box load of X, one of the
 //            P rows (positions of a tile are consecutive) and one of the 64 x k slice of U.
-//   warp 1   one thread issues tcgen05.mma (M=128, N=k rounded up to 16, K=16) for the stage and
-//            commits to the stage's "empty" barrier; the last stage of a tile also commits to the
-//            accumulator's "full" barrier.  This warp owns the TMEM allocation.
+//   warps 1, 10, 11  one thread each issues the tcgen05.mma (M=128, N=k rounded up to 16, K=16) of
+//            ONE A operand (X, E, P) into its own accumulator and commits to the stage's "empty"
+//            barrier; a single thread issues only one such instruction per ~85 clocks, three
+//            issue side by side.  The last stage of a tile also commits to the accumulators'
+//            "full" barrier.  Warp 1 owns the TMEM allocation.
 //   warps 2-5  gather the E rows of the tile: 8 lanes copy one 128-byte row piece with cp.async
 //            straight into the swizzled tile, three stages ahead of the barrier arrival that
 //            publishes them (an id outside the table points at a row of zeros).
@@ -28,7 +30,7 @@
 
 namespace ssn {
 
-constexpr int kUmmaThreads = 320;
+constexpr int kUmmaThreads = 384;
 constexpr int kUmmaTile = 128;     // tokens per tile (MMA M)
 constexpr int kUmmaCols = 64;      // columns of X per stage (one 128-byte swizzle row)
 constexpr int kWaitSpins = 1 << 22;
@@ -128,6 +130,10 @@ struct UmmaProjectConfig {
   static_assert(kStagesN >= 2, "no room for two stages");
   static constexpr int kGatherLag = kStagesN > 3 ? 3 : kStagesN - 1;   // stages between issuing a gather and publishing it
   static constexpr int kAccCols = kN <= 32 ? 32 : (kN <= 64 ? 64 : 128);   // TMEM columns per accumulator
+  static constexpr int kIssuers = kATiles;                          // one MMA-issuing thread per A operand
+  static constexpr int kBufs = 2 * kIssuers * kAccCols <= 512 ? 2 : 1;   // accumulator sets (tiles in flight)
+  static constexpr int kTmemCols = (kBufs * kIssuers * kAccCols) <= 128 ? 128 : ((kBufs * kIssuers * kAccCols) <= 256 ? 256 : 512);
+  static_assert(kBufs * kIssuers * kAccCols <= 512, "accumulators do not fit in tensor memory");
   static constexpr int kBarBytes = (2 * kStagesN + 4) * 8 + 16;
   static constexpr int kSmemBytes = 1024 + kStagesN * kStageBytes + kBarBytes;
 };
@@ -160,17 +166,17 @@ codec_umma_project_kernel(const MmaArgs a, const __grid_constant__ UmmaMaps maps
   if (threadIdx.x == 0) {
     for (int s = 0; s < S; ++s) {
       mbar_init(full_bar(s), HAS_E ? 5 : 1);
-      mbar_init(empty_bar(s), 1);
+      mbar_init(empty_bar(s), Cfg::kIssuers);
     }
     for (int b = 0; b < 2; ++b) {
-      mbar_init(acc_full_bar(b), 1);
+      mbar_init(acc_full_bar(b), Cfg::kIssuers);
       mbar_init(acc_empty_bar(b), 4);
     }
     asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
   }
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(tmem_slot),
-                 "r"(2 * Cfg::kAccCols) : "memory");
+                 "r"(Cfg::kTmemCols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
   }
   asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
@@ -210,39 +216,37 @@ codec_umma_project_kernel(const MmaArgs a, const __grid_constant__ UmmaMaps maps
         }
       }
     }
-  } else if (warp == 1) {
-    // ------------------------------------------------------------------------- MMA issuer
-    if (lane == 0) {
-      constexpr uint32_t idesc_pos = umma_idesc(Cfg::kN, false), idesc_neg = umma_idesc(Cfg::kN, true);
+  } else if (warp == 1 || warp >= 10) {
+    // ------------------------------------------------------------------------- MMA issuers
+    // One thread per A operand (X: warp 1, E: warp 10, P: warp 11), each with its own
+    // accumulator, so that the three instruction streams issue side by side; the epilogue
+    // combines X.U - E.U - P.U.  A stage is released when all issuers have committed.
+    // warp 1 -> X; warp 10 -> the first table operand present; warp 11 -> P when both are present
+    const int which = warp == 1 ? 0 : (warp == 10 ? (Cfg::kATiles >= 2 ? 1 : -1) : (warp == 11 && Cfg::kATiles == 3 ? 2 : -1));
+    if (lane == 0 && which >= 0) {
+      constexpr uint32_t idesc = umma_idesc(Cfg::kN, false);
       int slot = 0;
       uint32_t parity = 0;
       int64_t tcount = 0;
       for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x, ++tcount) {
-        const int buf = (int)(tcount & 1);
-        const uint32_t acc_parity = (uint32_t)((tcount >> 1) & 1);
+        const int buf = (int)(tcount % Cfg::kBufs);
+        const uint32_t acc_parity = (uint32_t)((tcount / Cfg::kBufs) & 1);
         if (!dead && !mbar_wait(acc_empty_bar(buf), acc_parity ^ 1u)) timed_out();
         asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
-        const uint32_t d_tmem = tmem_base + (uint32_t)buf * Cfg::kAccCols;
+        const uint32_t d_tmem = tmem_base + (uint32_t)(buf * Cfg::kIssuers + which) * Cfg::kAccCols;
         for (int st = 0; st < nstage; ++st) {
           if (!dead && !mbar_wait(full_bar(slot), parity)) timed_out();
           asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
           const uint32_t base = smem0 + (uint32_t)slot * Cfg::kStageBytes;
+          const uint32_t abase = base + (uint32_t)which * Cfg::kATileBytes;
           const uint32_t ubase = base + Cfg::kATiles * Cfg::kATileBytes;
 #pragma unroll
           for (int j = 0; j < kUmmaCols / 16; ++j) {
             // U slice: rows are the contracted index (16 rows = 2048 bytes per K step), 64-column
             // groups kUGroupBytes apart, 8-row groups 1024 bytes apart
             const uint64_t bdesc = umma_desc(ubase + j * 2048, Cfg::kUGroupBytes, 1024, 2);
-            const uint64_t xdesc = umma_desc(base + j * 32, 16, 1024, 2);
-            umma_bf16(d_tmem, xdesc, bdesc, idesc_pos, (st > 0 || j > 0) ? 1u : 0u);
-            if (HAS_E) {
-              const uint64_t edesc = umma_desc(base + kETile * Cfg::kATileBytes + j * 32, 16, 1024, 2);
-              umma_bf16(d_tmem, edesc, bdesc, idesc_neg, 1u);
-            }
-            if (HAS_P) {
-              const uint64_t pdesc = umma_desc(base + kPTile * Cfg::kATileBytes + j * 32, 16, 1024, 2);
-              umma_bf16(d_tmem, pdesc, bdesc, idesc_neg, 1u);
-            }
+            const uint64_t adesc = umma_desc(abase + j * 32, 16, 1024, 2);
+            umma_bf16(d_tmem, adesc, bdesc, idesc, (st > 0 || j > 0) ? 1u : 0u);
           }
           umma_commit(empty_bar(slot));
           if (st == nstage - 1) umma_commit(acc_full_bar(buf));
@@ -306,15 +310,27 @@ codec_umma_project_kernel(const MmaArgs a, const __grid_constant__ UmmaMaps maps
     int64_t tcount = 0;
     const bool vec = ((a.ldzout & 7) == 0) && ((reinterpret_cast<uintptr_t>(a.zout) & 15) == 0);
     for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x, ++tcount) {
-      const int buf = (int)(tcount & 1);
-      const uint32_t acc_parity = (uint32_t)((tcount >> 1) & 1);
+      const int buf = (int)(tcount % Cfg::kBufs);
+      const uint32_t acc_parity = (uint32_t)((tcount / Cfg::kBufs) & 1);
       if (!dead && !mbar_wait(acc_full_bar(buf), acc_parity)) timed_out();
       asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
-      const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)buf * Cfg::kAccCols;
+      const uint32_t taddr =
+          tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * Cfg::kIssuers) * Cfg::kAccCols;
       uint32_t v[Cfg::kN / 16][16];
 #pragma unroll
       for (int q = 0; q < Cfg::kN / 16; ++q) tmem_ld16(taddr + q * 16, v[q]);
       asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
+#pragma unroll
+      for (int op = 1; op < Cfg::kIssuers; ++op) {   // Z = X.U - E.U - P.U
+#pragma unroll
+        for (int q = 0; q < Cfg::kN / 16; ++q) {
+          uint32_t w[16];
+          tmem_ld16(taddr + op * Cfg::kAccCols + q * 16, w);
+          asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
+#pragma unroll
+          for (int i = 0; i < 16; ++i) v[q][i] = __float_as_uint(__uint_as_float(v[q][i]) - __uint_as_float(w[i]));
+        }
+      }
       asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
       __syncwarp();
       if (lane == 0) mbar_arrive(acc_empty_bar(buf));
@@ -350,7 +366,7 @@ codec_umma_project_kernel(const MmaArgs a, const __grid_constant__ UmmaMaps maps
   if (warp == 1) {
     asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem_base),
-                 "r"(2 * Cfg::kAccCols) : "memory");
+                 "r"(Cfg::kTmemCols) : "memory");
   }
 }
 
