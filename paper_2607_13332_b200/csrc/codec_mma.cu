@@ -3,6 +3,7 @@
 #include "codec_mma_dsplit.cuh"
 #include "codec_expand64.cuh"
 #include "codec_umma.cuh"
+#include "codec_umma_roundtrip.cuh"
 
 
 #include "codec_mma_launch.h"
@@ -196,6 +197,8 @@ cudaError_t launch_codec_umma_project(const MmaArgs &a, bool shift, int sm_count
   UmmaMaps maps;
   if (!make_sw128_map(&maps.x, a.src, a.n, a.d, a.lds, kUmmaTile)) return cudaErrorNotSupported;
   if (!make_sw128_map(&maps.u, a.U, a.d, a.k, a.ldu, kUmmaCols)) return cudaErrorNotSupported;
+  if (!make_sw128_map(&maps.u_wide, a.U, a.d, a.k <= 64 ? 64 : 128, a.ldu, kUmmaCols))
+    return cudaErrorNotSupported;
   maps.p = maps.x;
   if (has_p && !make_sw128_map(&maps.p, a.shift.P, a.shift.max_pos, a.d, a.shift.ldp, kUmmaTile))
     return cudaErrorNotSupported;
@@ -207,6 +210,43 @@ cudaError_t launch_codec_umma_project(const MmaArgs &a, bool shift, int sm_count
   return launch_umma_ntp<16>(a, has_e, has_p, maps, sm_count, stream);
 }
 
+namespace {
+template <int NTP>
+cudaError_t launch_roundtrip_ntp(const MmaArgs &a, const UmmaRoundTripMaps &maps, int sm_count, cudaStream_t stream) {
+  auto kernel = codec_umma_roundtrip_kernel<NTP>;
+  constexpr int smem = UmmaRoundTripConfig<NTP>::kSmemBytes;
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  int64_t grid = (a.n + kUmmaTile - 1) / kUmmaTile;
+  if (grid > sm_count) grid = sm_count;
+  kernel<<<(unsigned)grid, kRoundTripThreads, smem, stream>>>(a, maps);
+  return cudaGetLastError();
+}
+}  // namespace
+
+// Project-then-expand on tcgen05 (weight re-projection, projected gradient).  Returns
+// cudaErrorNotSupported when the call should take the mma.sync kernels instead: k > 64, d not
+// a multiple of 128, few rows, no tensor map (unaligned base or leading dimension).
+cudaError_t launch_codec_umma_roundtrip(const MmaArgs &a, int sm_count, cudaStream_t stream) {
+  if (a.src == nullptr || a.dst == nullptr) return cudaErrorNotSupported;
+  if (a.d % kChunkCols != 0 || a.k > 64 || a.n < 4 * kUmmaTile || a.n > 0x7fffffffLL)
+    return cudaErrorNotSupported;
+  UmmaRoundTripMaps maps;
+  if (!make_sw128_map(&maps.s, a.src, a.n, a.d, a.lds, kUmmaTile)) return cudaErrorNotSupported;
+  if (!make_sw128_map(&maps.u, a.U, a.d, a.k, a.ldu, kUmmaCols)) return cudaErrorNotSupported;
+  if (!make_sw128_map(&maps.u_wide, a.U, a.d, 64, a.ldu, kUmmaCols)) return cudaErrorNotSupported;
+  if (!make_sw128_map(&maps.out, a.dst, a.n, a.d, a.lddst, 32)) return cudaErrorNotSupported;
+  const int ntp = 2 * ((a.k + 15) / 16);
+  if (ntp <= 2) return launch_roundtrip_ntp<2>(a, maps, sm_count, stream);
+  if (ntp <= 4) return launch_roundtrip_ntp<4>(a, maps, sm_count, stream);
+  if (ntp <= 6) return launch_roundtrip_ntp<6>(a, maps, sm_count, stream);
+  return launch_roundtrip_ntp<8>(a, maps, sm_count, stream);
+}
+
 bool codec_mma_supports(int d, int k) {
   return d % 32 == 0 && (int64_t)d * 2 <= kZeroRowBytes && k >= 1 && k <= 128;
 }
@@ -215,6 +255,10 @@ cudaError_t launch_codec_mma(const MmaArgs &a, bool shift, int mode, int sm_coun
                              cudaStream_t stream) {
   if (mode == kModeProject) {
     cudaError_t e = launch_codec_umma_project(a, shift, sm_count, stream);
+    if (e != cudaErrorNotSupported) return e;
+  }
+  if (mode == (kModeProject | kModeExpand) && !shift) {
+    cudaError_t e = launch_codec_umma_roundtrip(a, sm_count, stream);
     if (e != cudaErrorNotSupported) return e;
   }
   const int nt = (a.k + 7) / 8;

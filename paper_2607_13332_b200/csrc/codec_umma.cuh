@@ -2,16 +2,16 @@
 //     Z = X U - E[ids] U - P[pos] U        compress (SHIFT) / grad-project coefficients (!SHIFT)
 //
 // The subtraction of Eq. (ssn_compress) is moved through the contraction: the three products
-// are accumulated into one fp32 accumulator in tensor memory, the E and P products with the
-// instruction descriptor's negate-A bit set.  bf16 x bf16 products are exact in fp32, so the
-// only rounding is fp32 accumulation, and no thread ever touches an element of X, E or P:
+// X U, E U and P U are accumulated in fp32 in tensor memory and combined in the epilogue.
+// bf16 x bf16 products are exact in fp32, so the only rounding is fp32 accumulation, and no
+// thread ever touches an element of X, E or P:
 //
 //   warp 0   producer.  Per stage (128 tokens x 64 columns) one TMA box load of X, one of the
 //            P rows (positions of a tile are consecutive) and one of the 64 x k slice of U.
 //   warps 1, 10, 11  one thread each issues the tcgen05.mma (M=128, N=k rounded up to 16, K=16) of
 //            ONE A operand (X, E, P) into its own accumulator and commits to the stage's "empty"
-//            barrier; a single thread issues only one such instruction per ~85 clocks, three
-//            issue side by side.  The last stage of a tile also commits to the accumulators'
+//            barrier (the tensor pipe retires one such instruction per ~87 clocks whatever
+//            its N).  The last stage of a tile also commits to the accumulators'
 //            "full" barrier.  Warp 1 owns the TMEM allocation.
 //   warps 2-5  gather the E rows of the tile: 8 lanes copy one 128-byte row piece with cp.async
 //            straight into the swizzled tile, three stages ahead of the barrier arrival that
@@ -126,7 +126,7 @@ struct UmmaProjectConfig {
   static constexpr int kTmaBytes = kStageBytes - (HAS_E ? kATileBytes : 0);
   static constexpr int kMaxSmem = 227 * 1024;
   static constexpr int kFit = (kMaxSmem - 1024 - 512) / kStageBytes;
-  static constexpr int kStagesN = kFit < 8 ? kFit : 8;
+  static constexpr int kStagesN = kFit < 10 ? kFit : 10;
   static_assert(kStagesN >= 2, "no room for two stages");
   static constexpr int kGatherLag = kStagesN > 3 ? 3 : kStagesN - 1;   // stages between issuing a gather and publishing it
   static constexpr int kAccCols = kN <= 32 ? 32 : (kN <= 64 ? 64 : 128);   // TMEM columns per accumulator
@@ -138,8 +138,13 @@ struct UmmaProjectConfig {
   static constexpr int kSmemBytes = 1024 + kStagesN * kStageBytes + kBarBytes;
 };
 
+// u describes U as it is ([d x k]: a 64-column box that reaches past column k is filled with
+// zeros, which the TMA unit does slowly); u_wide claims 64 (128) columns per row with the same
+// row pitch, so that a box never leaves the tensor: the columns past k then hold the start of
+// the following rows, and feed only accumulator columns that are never stored.  u_wide is used
+// for all stages but the last one of U, whose box would read past the end of the buffer.
 struct UmmaMaps {
-  CUtensorMap x, p, u;
+  CUtensorMap x, p, u, u_wide;
 };
 
 template <int NTP, bool HAS_E, bool HAS_P>
@@ -206,8 +211,8 @@ codec_umma_project_kernel(const MmaArgs a, const __grid_constant__ UmmaMaps maps
           if (HAS_P) tma_load_2d(base + kPTile * Cfg::kATileBytes, &maps.p, bar, st * kUmmaCols, pos0);
 #pragma unroll
           for (int ug = 0; ug < Cfg::kUGroups; ++ug)
-            tma_load_2d(base + Cfg::kATiles * Cfg::kATileBytes + ug * Cfg::kUGroupBytes, &maps.u, bar, ug * 64,
-                        st * kUmmaCols);
+            tma_load_2d(base + Cfg::kATiles * Cfg::kATileBytes + ug * Cfg::kUGroupBytes,
+                        st == nstage - 1 ? &maps.u : &maps.u_wide, bar, ug * 64, st * kUmmaCols);
         }
         __syncwarp();
         if (++slot == S) {
@@ -225,6 +230,9 @@ codec_umma_project_kernel(const MmaArgs a, const __grid_constant__ UmmaMaps maps
     const int which = warp == 1 ? 0 : (warp == 10 ? (Cfg::kATiles >= 2 ? 1 : -1) : (warp == 11 && Cfg::kATiles == 3 ? 2 : -1));
     if (lane == 0 && which >= 0) {
       constexpr uint32_t idesc = umma_idesc(Cfg::kN, false);
+      // A tiles: K-major rows of 128 bytes, 8-row groups 1024 bytes apart.  U slice: MN-major,
+      // 64-column groups kUGroupBytes apart, 8-row groups 1024 bytes apart.
+      const uint64_t adesc0 = umma_desc(0, 16, 1024, 2), bdesc0 = umma_desc(0, Cfg::kUGroupBytes, 1024, 2);
       int slot = 0;
       uint32_t parity = 0;
       int64_t tcount = 0;
@@ -238,16 +246,13 @@ codec_umma_project_kernel(const MmaArgs a, const __grid_constant__ UmmaMaps maps
           if (!dead && !mbar_wait(full_bar(slot), parity)) timed_out();
           asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
           const uint32_t base = smem0 + (uint32_t)slot * Cfg::kStageBytes;
-          const uint32_t abase = base + (uint32_t)which * Cfg::kATileBytes;
-          const uint32_t ubase = base + Cfg::kATiles * Cfg::kATileBytes;
+          // the start-address field (address / 16) is added to descriptors built once: a K step
+          // is 32 bytes of an A row and 16 rows = 2048 bytes of the U slice
+          const uint64_t adesc = adesc0 + ((base + (uint32_t)which * Cfg::kATileBytes) >> 4);
+          const uint64_t bdesc = bdesc0 + ((base + Cfg::kATiles * Cfg::kATileBytes) >> 4);
 #pragma unroll
-          for (int j = 0; j < kUmmaCols / 16; ++j) {
-            // U slice: rows are the contracted index (16 rows = 2048 bytes per K step), 64-column
-            // groups kUGroupBytes apart, 8-row groups 1024 bytes apart
-            const uint64_t bdesc = umma_desc(ubase + j * 2048, Cfg::kUGroupBytes, 1024, 2);
-            const uint64_t adesc = umma_desc(abase + j * 32, 16, 1024, 2);
-            umma_bf16(d_tmem, adesc, bdesc, idesc, (st > 0 || j > 0) ? 1u : 0u);
-          }
+          for (int j = 0; j < kUmmaCols / 16; ++j)
+            umma_bf16(d_tmem, adesc + j * 2, bdesc + j * 128, idesc, (st > 0 || j > 0) ? 1u : 0u);
           umma_commit(empty_bar(slot));
           if (st == nstage - 1) umma_commit(acc_full_bar(buf));
           if (++slot == S) {
