@@ -4,6 +4,7 @@
 #include "codec_expand64.cuh"
 #include "codec_umma.cuh"
 #include "codec_umma_roundtrip.cuh"
+#include "codec_umma_expand.cuh"
 
 
 #include "codec_mma_launch.h"
@@ -155,6 +156,37 @@ bool make_sw128_map(CUtensorMap *map, const void *base, int64_t rows, int64_t co
             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Row-major bf16 tensor [n2][n1][cols] (row pitch ld, slab pitch ld2, in elements), fetched in
+// boxes of 64 columns x box1 x box2 into the 128-byte swizzled layout.
+bool make_sw128_map3(CUtensorMap *map, const void *base, int64_t cols, int64_t n1, int64_t n2, int64_t ld,
+                     int64_t ld2, int box1, int box2) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (fn == nullptr || n1 < 1 || n2 < 1 || n1 > 0x7fffffffLL || n2 > 0x7fffffffLL) return false;
+  cuuint64_t dims[3] = {(cuuint64_t)cols, (cuuint64_t)n1, (cuuint64_t)n2};
+  cuuint64_t strides[2] = {(cuuint64_t)ld * 2, (cuuint64_t)ld2 * 2};
+  cuuint32_t box[3] = {(cuuint32_t)kUmmaCols, (cuuint32_t)box1, (cuuint32_t)box2};
+  cuuint32_t estr[3] = {1, 1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box,
+            estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <bool HAS_E, bool HAS_P>
+cudaError_t launch_umma_expand_one(const MmaArgs &a, const ExpandGeometry &geo, const UmmaExpandMaps &maps,
+                                   int sm_count, cudaStream_t stream) {
+  auto kernel = codec_umma_expand_kernel<HAS_E, HAS_P>;
+  constexpr int smem = UmmaExpandConfig<HAS_E, HAS_P>::kSmemBytes;
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  int64_t grid = geo.ntiles < sm_count ? geo.ntiles : sm_count;
+  kernel<<<(unsigned)grid, kExpandThreads, smem, stream>>>(a, geo, maps);
+  return cudaGetLastError();
+}
+
 template <int NTP, bool HAS_E, bool HAS_P>
 cudaError_t launch_umma_one(const MmaArgs &a, const UmmaMaps &maps, int sm_count, cudaStream_t stream) {
   auto kernel = codec_umma_project_kernel<NTP, HAS_E, HAS_P>;
@@ -247,6 +279,54 @@ cudaError_t launch_codec_umma_roundtrip(const MmaArgs &a, int sm_count, cudaStre
   return launch_roundtrip_ntp<8>(a, maps, sm_count, stream);
 }
 
+// Expansion (decompress) on tcgen05.  Returns cudaErrorNotSupported when the call should take the
+// mma.sync kernel instead: k > 64, d not a multiple of 128, few tokens, no tensor map, or a
+// position table with explicit positions / a batch that is not made of groups of 8 whole
+// sequences whose length is a multiple of 16.
+cudaError_t launch_codec_umma_expand(const MmaArgs &a, bool shift, int sm_count, cudaStream_t stream) {
+  if (a.zin == nullptr || a.dst == nullptr || a.src != nullptr) return cudaErrorNotSupported;
+  if (a.d % kChunkCols != 0 || a.k > 64 || a.n < 4 * kUmmaTile || a.n > 0x7fffffffLL)
+    return cudaErrorNotSupported;
+  const bool has_e = shift && a.shift.E != nullptr, has_p = shift && a.shift.P != nullptr;
+  ExpandGeometry geo{};
+  geo.seq_len = a.shift.seq_len;
+  if (has_p) {
+    const int64_t L = a.shift.seq_len;
+    if (a.shift.pos != nullptr || L < kGridPos || L % kGridPos != 0 || L > a.shift.max_pos || a.n % L != 0 ||
+        (a.n / L) % kGridSeqs != 0)
+      return cudaErrorNotSupported;
+    geo.grid_mode = 1;
+    geo.nsg = (int32_t)(a.n / L / kGridSeqs);
+    geo.ntiles = (int64_t)geo.nsg * (L / kGridPos);
+  } else {
+    geo.grid_mode = 0;
+    geo.nsg = 1;
+    geo.ntiles = (a.n + kUmmaTile - 1) / kUmmaTile;
+  }
+  UmmaExpandMaps maps;
+  if (geo.grid_mode) {
+    const int64_t L = a.shift.seq_len, B = a.n / L;
+    if (!make_sw128_map3(&maps.z, a.zin, a.k, L, B, a.ldzin, L * a.ldzin, kGridPos, kGridSeqs))
+      return cudaErrorNotSupported;
+    if (!make_sw128_map3(&maps.out, a.dst, a.d, L, B, a.lddst, L * a.lddst, kGridPos, 32 / kGridPos))
+      return cudaErrorNotSupported;
+    if (!make_sw128_map(&maps.p, a.shift.P, a.shift.max_pos, a.d, a.shift.ldp, kGridPos))
+      return cudaErrorNotSupported;
+  } else {
+    if (!make_sw128_map3(&maps.z, a.zin, a.k, a.n, 1, a.ldzin, a.n * a.ldzin, kUmmaTile, 1))
+      return cudaErrorNotSupported;
+    if (!make_sw128_map3(&maps.out, a.dst, a.d, a.n, 1, a.lddst, a.n * a.lddst, 32, 1))
+      return cudaErrorNotSupported;
+    maps.p = maps.z;
+  }
+  if (!make_sw128_map(&maps.u, a.U, a.d, a.k, a.ldu, kUmmaCols)) return cudaErrorNotSupported;
+  if (!make_sw128_map(&maps.u_wide, a.U, a.d, 64, a.ldu, kUmmaCols)) return cudaErrorNotSupported;
+  if (has_e && has_p) return launch_umma_expand_one<true, true>(a, geo, maps, sm_count, stream);
+  if (has_e) return launch_umma_expand_one<true, false>(a, geo, maps, sm_count, stream);
+  if (has_p) return launch_umma_expand_one<false, true>(a, geo, maps, sm_count, stream);
+  return launch_umma_expand_one<false, false>(a, geo, maps, sm_count, stream);
+}
+
 bool codec_mma_supports(int d, int k) {
   return d % 32 == 0 && (int64_t)d * 2 <= kZeroRowBytes && k >= 1 && k <= 128;
 }
@@ -270,7 +350,9 @@ cudaError_t launch_codec_mma(const MmaArgs &a, bool shift, int mode, int sm_coun
                                         : launch_dsplit<1>(a, shift, mode, nt, sm_count, stream);
   }
   if (!small && mode == kModeExpand) {
-    cudaError_t e = launch_expand64(a, shift, sm_count, stream);
+    cudaError_t e = launch_codec_umma_expand(a, shift, sm_count, stream);
+    if (e != cudaErrorNotSupported) return e;
+    e = launch_expand64(a, shift, sm_count, stream);
     if (e != cudaErrorNotSupported) return e;
   }
   if (small) {

@@ -1,0 +1,384 @@
+// tcgen05 / TMA expansion kernel of the SSN codec (bf16, sm_100a), k <= 64:
+//     Xhat = Z U^T + E[ids] + P[pos]          decompress (receiver side of Eq. ssn_compress)
+//
+// A tile is 128 tokens, a chunk 128 output columns accumulated in 128 TMEM columns:
+//     D  = Z_tile[128 x k] * (U rows of the chunk)^T     ceil(k/16) MMAs (M=128, N=128, K=16)
+//     D += Sel[128 x 16]   * P_rows[16 x 128]            one MMA, see below
+// and the epilogue adds the gathered E rows in fp32 before the single rounding to bf16.
+//
+// Positions.  With implicit positions (t mod seq_len) a tile is laid out as 8 sequences x 16
+// consecutive positions (a 3-D TMA box), so it needs only 16 rows of P, which enter the
+// accumulator through a constant 0/1 selection matrix (row r selects position r mod 16):
+// 1.0 * bf16 is exact and the sum is taken in fp32, so P costs one MMA per chunk and no thread
+// touches it.  Without P a tile is 128 consecutive tokens.
+//
+//   warp 0     producer: per tile the Z tile; per chunk the 128 rows of U (K-major operand)
+//              and the 16 rows of P.
+//   warp 1     MMA issuer (one thread), owns the TMEM allocation; two accumulators alternate.
+//   warps 2-9  epilogue, two groups of four that take alternate chunks: tcgen05.ld one token
+//              row per thread, add the E row piece from shared memory, round to bf16 into a
+//              swizzled staging slab and hand 32 rows x 64 columns to a TMA store (which also
+//              clips the rows past n).
+//   warps 10-13  gather the E rows of the tile, 64 columns at a time, with cp.async into
+//              swizzled stages (an id outside the table points at a row of zeros); the epilogue
+//              forms the sum in place and the stage is the source of the TMA store.
+// Every wait is bounded; a wait that runs out sets SSN_DEV_TIMEOUT and the kernel still ends.
+#pragma once
+
+#include "codec_umma_roundtrip.cuh"
+
+namespace ssn {
+
+constexpr int kExpandThreads = 448;
+constexpr int kGatherWarps = 4;
+constexpr int kGridSeqs = 8, kGridPos = 16;   // tile shape with implicit positions
+
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, uint32_t bar,
+                                            int c0, int c1, int c2) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cta.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];\n"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap *map, uint32_t src, int c0, int c1, int c2) {
+  asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];\n"
+               ::"l"(map), "r"(src), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+
+template <bool HAS_E, bool HAS_P>
+struct UmmaExpandConfig {
+  static constexpr int kTileBytes = kUmmaTile * 128;            // [128 rows x 128 B]
+  static constexpr int kU2Bytes = kChunkCols * 128;             // 128 rows of U, K-major
+  static constexpr int kPBytes = HAS_P ? 2 * kGridPos * 128 : 0;   // 16 rows of P, two 64-column groups
+  static constexpr int kUStageBytes = kU2Bytes + kPBytes;
+  static constexpr int kUStages = 3;
+  static constexpr int kEStageBytes = kTileBytes;               // E rows of 64 columns of a chunk
+  // Without E the epilogue warps stage their output in two [32 x 128 B] slabs each; with E the
+  // sum is formed in place in the E stage, which is then the source of the TMA store.
+  static constexpr int kStagingBytes = HAS_E ? 0 : 8 * 2 * 4096;
+  static constexpr int kFixedBytes =
+      2 * kTileBytes + (HAS_P ? kTileBytes : 0) + kUStages * kUStageBytes + kStagingBytes;
+  static constexpr int kMaxSmem = 227 * 1024;
+  static constexpr int kEFit = (kMaxSmem - 1024 - 512 - kFixedBytes) / kEStageBytes;
+  static constexpr int kEStages = HAS_E ? (kEFit < 8 ? kEFit : 8) : 0;
+  static_assert(!HAS_E || kEStages >= 4, "no room for the E ring");
+  static constexpr int kTmemCols = 256;
+  static constexpr int SE = HAS_E ? kEStages : 1;
+  static constexpr int kBars = 4 + 2 * kUStages + 2 * SE + 4;
+  static constexpr int kSmemBytes = 1024 + kFixedBytes + kEStages * kEStageBytes + kBars * 8 + 16;
+};
+
+struct UmmaExpandMaps {
+  // z: Z tile (box 64 x 128 rows, or 64 x 16 x 8); u / u_wide: 64 x 64 boxes of U (see UmmaMaps);
+  // p: 64 columns x 16 rows of P; out: 64 columns x 32 rows (or 64 x 16 x 2)
+  CUtensorMap z, u, u_wide, p, out;
+};
+
+struct ExpandGeometry {
+  int32_t grid_mode;      // 1: tiles of 8 sequences x 16 positions, 0: 128 consecutive tokens
+  int32_t seq_len;
+  int32_t nsg;            // groups of 8 sequences
+  int64_t ntiles;
+};
+
+template <bool HAS_E, bool HAS_P>
+__global__ void __launch_bounds__(kExpandThreads, 1)
+codec_umma_expand_kernel(const MmaArgs a, const ExpandGeometry geo, const __grid_constant__ UmmaExpandMaps maps) {
+  using Cfg = UmmaExpandConfig<HAS_E, HAS_P>;
+  constexpr int SU = Cfg::kUStages, SE = Cfg::SE;
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int nchunks = a.d / kChunkCols;
+  const int ksteps = (a.k + 15) / 16;
+  const int64_t ntiles = geo.ntiles;
+
+  const uint32_t smem0 = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t z_base = smem0;                                         // two Z tiles
+  const uint32_t sel = z_base + 2 * Cfg::kTileBytes;                     // selection matrix (HAS_P)
+  const uint32_t u_ring = sel + (HAS_P ? Cfg::kTileBytes : 0);
+  const uint32_t staging = u_ring + SU * Cfg::kUStageBytes;
+  const uint32_t e_ring = staging + Cfg::kStagingBytes;
+  const uint32_t bars = e_ring + Cfg::kEStages * Cfg::kEStageBytes;
+  auto z_full_bar = [&](int b) { return bars + b * 8; };
+  auto z_empty_bar = [&](int b) { return bars + (2 + b) * 8; };
+  auto u_full_bar = [&](int s) { return bars + (4 + s) * 8; };
+  auto u_empty_bar = [&](int s) { return bars + (4 + SU + s) * 8; };
+  auto e_full_bar = [&](int s) { return bars + (4 + 2 * SU + s) * 8; };
+  auto e_empty_bar = [&](int s) { return bars + (4 + 2 * SU + SE + s) * 8; };
+  auto d_full_bar = [&](int b) { return bars + (4 + 2 * SU + 2 * SE + b) * 8; };
+  auto d_empty_bar = [&](int b) { return bars + (4 + 2 * SU + 2 * SE + 2 + b) * 8; };
+  const uint32_t tmem_slot = bars + Cfg::kBars * 8;
+  volatile uint32_t *tmem_slot_ptr =
+      reinterpret_cast<volatile uint32_t *>(smem_raw + (tmem_slot - smem_u32(smem_raw)));
+
+  if (HAS_P) {
+    // Sel[r][j] = 1 for j == r mod 16 (K-major, 128-byte rows, swizzled); only K = 16 is read
+    for (uint32_t i = threadIdx.x; i < Cfg::kTileBytes / 16; i += blockDim.x) {
+      const uint32_t r = i >> 3, c = i & 7;     // row, logical 16-byte piece
+      uint4 v = make_uint4(0, 0, 0, 0);
+      const uint32_t j = r & 15;
+      if (c == (j >> 3)) {
+        const uint32_t e = j & 7, word = 0x3F80u << ((e & 1) * 16);
+        if ((e >> 1) == 0) v.x = word;
+        if ((e >> 1) == 1) v.y = word;
+        if ((e >> 1) == 2) v.z = word;
+        if ((e >> 1) == 3) v.w = word;
+      }
+      const uint32_t off = r * 128 + ((c ^ (r & 7)) << 4);
+      *reinterpret_cast<uint4 *>(smem_raw + (sel - smem_u32(smem_raw)) + off) = v;
+    }
+    asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
+  }
+  if (threadIdx.x == 0) {
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(z_full_bar(b), 1);
+      mbar_init(z_empty_bar(b), 1);
+      mbar_init(d_full_bar(b), 1);
+      mbar_init(d_empty_bar(b), 4);
+    }
+    for (int s = 0; s < SU; ++s) {
+      mbar_init(u_full_bar(s), 1);
+      mbar_init(u_empty_bar(s), 1);
+    }
+    for (int s = 0; s < SE; ++s) {
+      mbar_init(e_full_bar(s), kGatherWarps * 32);   // one arrival per gather thread
+      mbar_init(e_empty_bar(s), 4);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(tmem_slot),
+                 "r"(Cfg::kTmemCols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+  const uint32_t tmem_base = *tmem_slot_ptr;
+  bool dead = false;
+  auto timed_out = [&]() {
+    dead = true;
+    if (a.shift.dev_status) atomicOr(a.shift.dev_status, SSN_DEV_TIMEOUT);
+  };
+  // tile -> TMA coordinates (row coordinate, sequence coordinate) of its first token
+  auto tile_coords = [&](int64_t tile, int &c1, int &c2) {
+    if (geo.grid_mode) {
+      const int64_t pb = tile / geo.nsg;
+      c1 = (int)pb * kGridPos;
+      c2 = (int)(tile - pb * geo.nsg) * kGridSeqs;
+    } else {
+      c1 = (int)(tile * kUmmaTile);
+      c2 = 0;
+    }
+  };
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------------- producer
+    int slot = 0;
+    uint32_t parity = 1;
+    int64_t tcount = 0;
+    for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x, ++tcount) {
+      int c1, c2;
+      tile_coords(tile, c1, c2);
+      const int zb = (int)(tcount & 1);
+      if (!dead && !mbar_wait(z_empty_bar(zb), (uint32_t)(((tcount >> 1) & 1) ^ 1))) timed_out();
+      if (lane == 0) {
+        mbar_expect_tx(z_full_bar(zb), Cfg::kTileBytes);
+        tma_load_3d(z_base + zb * Cfg::kTileBytes, &maps.z, z_full_bar(zb), 0, c1, c2);
+      }
+      for (int q = 0; q < nchunks; ++q) {
+        if (!dead && !mbar_wait(u_empty_bar(slot), parity)) timed_out();
+        const uint32_t base = u_ring + (uint32_t)slot * Cfg::kUStageBytes;
+        if (lane == 0) {
+          mbar_expect_tx(u_full_bar(slot), Cfg::kUStageBytes);
+          tma_load_2d(base, &maps.u_wide, u_full_bar(slot), 0, q * kChunkCols);
+          tma_load_2d(base + 8192, q == nchunks - 1 ? &maps.u : &maps.u_wide, u_full_bar(slot), 0,
+                      q * kChunkCols + 64);
+          if (HAS_P) {
+            tma_load_2d(base + Cfg::kU2Bytes, &maps.p, u_full_bar(slot), q * kChunkCols, c1);
+            tma_load_2d(base + Cfg::kU2Bytes + kGridPos * 128, &maps.p, u_full_bar(slot), q * kChunkCols + 64, c1);
+          }
+        }
+        __syncwarp();
+        if (++slot == SU) {
+          slot = 0;
+          parity ^= 1u;
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------------- MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc_kk = umma_idesc_kk(kChunkCols);            // Z tile x U chunk, both K-major
+      constexpr uint32_t idesc_kmn = umma_idesc(kChunkCols, false);       // Sel (K-major) x P rows (MN-major)
+      const uint64_t kdesc = umma_desc(0, 16, 1024, 2);
+      const uint64_t pdesc = umma_desc(0, kGridPos * 128, 1024, 2);       // 64-column groups 2048 bytes apart
+      const uint64_t seld = kdesc + (sel >> 4);
+      int slot = 0;
+      uint32_t parity = 0;
+      int64_t tcount = 0, ccount = 0;
+      for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x, ++tcount) {
+        const int zb = (int)(tcount & 1);
+        if (!dead && !mbar_wait(z_full_bar(zb), (uint32_t)((tcount >> 1) & 1))) timed_out();
+        const uint64_t zd = kdesc + ((z_base + zb * Cfg::kTileBytes) >> 4);
+        for (int q = 0; q < nchunks; ++q, ++ccount) {
+          const int db = (int)(ccount & 1);
+          if (!dead && !mbar_wait(d_empty_bar(db), (uint32_t)(((ccount >> 1) & 1) ^ 1))) timed_out();
+          if (!dead && !mbar_wait(u_full_bar(slot), parity)) timed_out();
+          asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+          const uint32_t base = u_ring + (uint32_t)slot * Cfg::kUStageBytes;
+          const uint32_t dacc = tmem_base + (uint32_t)db * kChunkCols;
+          const uint64_t bd = kdesc + (base >> 4);
+          for (int j = 0; j < ksteps; ++j) umma_bf16(dacc, zd + j * 2, bd + j * 2, idesc_kk, j > 0 ? 1u : 0u);
+          if (HAS_P) umma_bf16(dacc, seld, pdesc + ((base + Cfg::kU2Bytes) >> 4), idesc_kmn, 1u);
+          umma_commit(u_empty_bar(slot));
+          umma_commit(d_full_bar(db));
+          if (q == nchunks - 1) umma_commit(z_empty_bar(zb));
+          if (++slot == SU) {
+            slot = 0;
+            parity ^= 1u;
+          }
+        }
+      }
+    }
+  } else if (warp >= 10) {
+    // ------------------------------------------------------------------------- E row gather
+    // 8 lanes copy one 128-byte row piece with cp.async straight into the swizzled stage; the
+    // stage's "full" barrier counts one arrival per gather thread, made by the hardware when
+    // that thread's copies have landed, so nothing waits between issuing stages.
+    if (HAS_E) {
+      const int gw = warp - 10;                // rows 32*gw .. 32*gw+31 of the tile
+      const int piece = lane & 7, sub = lane >> 3;
+      int slot = 0;
+      uint32_t parity = 1;
+      for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+        int c1, c2;
+        tile_coords(tile, c1, c2);
+        const unsigned char *src[8];
+        uint32_t dst[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const int r = gw * 32 + i * 4 + sub;
+          const int64_t t = geo.grid_mode ? (int64_t)(c2 + r / kGridPos) * geo.seq_len + c1 + r % kGridPos
+                                          : (int64_t)c1 + r;
+          const int64_t er = t < a.n ? embedding_row(a.shift, t) : -1;
+          src[i] = (er >= 0 ? reinterpret_cast<const unsigned char *>(
+                                  static_cast<const __nv_bfloat16 *>(a.shift.E) + er * a.shift.lde)
+                            : g_zero_row) + piece * 16;
+          dst[i] = r * 128 + ((piece ^ (r & 7)) << 4);
+        }
+        for (int qg = 0; qg < 2 * nchunks; ++qg) {     // 64-column groups of the row
+          if (!dead && !mbar_wait(e_empty_bar(slot), parity)) timed_out();
+          const uint32_t base = e_ring + (uint32_t)slot * Cfg::kEStageBytes;
+#pragma unroll
+          for (int i = 0; i < 8; ++i) cp_async16(base + dst[i], src[i] + qg * 128, 16);
+          asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];\n" ::"r"(e_full_bar(slot)) : "memory");
+          if (++slot == SE) {
+            slot = 0;
+            parity ^= 1u;
+          }
+        }
+      }
+      cp_async_commit();
+      cp_async_wait<0>();
+    }
+  } else {
+    // ------------------------------------------------------------------------- epilogue
+    const int quarter = warp & 3;                 // TMEM lanes 32*quarter .. +31
+    const int group = warp >= 6 ? 1 : 0;          // takes the chunks with (chunk counter & 1) == group
+    const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16);
+    const uint32_t slab0 = staging + (uint32_t)(group * 4 + quarter) * 8192;   // !HAS_E: two slabs
+    int64_t ccount = 0;
+    int held = -1;                                // E stage whose store may still be reading it
+    for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+      int c1, c2;
+      tile_coords(tile, c1, c2);
+      // first token row of this warp's 32 rows, as TMA store coordinates
+      const int s1 = geo.grid_mode ? c1 : c1 + quarter * 32;
+      const int s2 = geo.grid_mode ? c2 + quarter * (32 / kGridPos) : 0;
+      const bool rows_live = geo.grid_mode || (int64_t)s1 < a.n;
+      for (int q = 0; q < nchunks; ++q, ++ccount) {
+        if ((int)(ccount & 1) != group) continue;
+        const int db = group;
+        if (!dead && !mbar_wait(d_full_bar(db), (uint32_t)((ccount >> 1) & 1))) timed_out();
+        asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+#pragma unroll
+        for (int g = 0; g < kChunkCols / 64; ++g) {
+          const int64_t ecount = 2 * ccount + g;
+          const int eslot = (int)(ecount % SE);
+          uint32_t v[4][16];
+#pragma unroll
+          for (int i = 0; i < 4; ++i) tmem_ld16(lane_addr + (uint32_t)db * kChunkCols + g * 64 + i * 16, v[i]);
+          asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
+          if (g == kChunkCols / 64 - 1) {
+            asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
+            __syncwarp();
+            if (lane == 0) mbar_arrive(d_empty_bar(db));
+          }
+          uint32_t slab;   // 32 rows x 128 B handed to the TMA store
+          if (HAS_E) {
+            if (!dead && !mbar_wait(e_full_bar(eslot), (uint32_t)((ecount / SE) & 1))) timed_out();
+            slab = e_ring + (uint32_t)eslot * Cfg::kEStageBytes + (uint32_t)quarter * 4096;
+          } else {
+            // the store that last read this slab (two stores ago) must be done reading it
+            if (lane == 0) bulk_wait_read<1>();
+            __syncwarp();
+            slab = slab0 + (uint32_t)g * 4096;
+          }
+          const uint32_t srow = slab + lane * 128;
+#pragma unroll
+          for (int c = 0; c < 8; ++c) {
+            const uint32_t *w = &v[c >> 1][(c & 1) * 8];
+            const uint32_t addr = srow + ((c ^ (lane & 7)) << 4);
+            float f[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) f[i] = __uint_as_float(w[i]);
+            if (HAS_E) {   // the sum replaces the E piece
+              uint32_t e0, e1, e2, e3;
+              asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];\n"
+                           : "=r"(e0), "=r"(e1), "=r"(e2), "=r"(e3) : "r"(addr));
+              f[0] += __uint_as_float(e0 << 16);
+              f[1] += __uint_as_float(e0 & 0xFFFF0000u);
+              f[2] += __uint_as_float(e1 << 16);
+              f[3] += __uint_as_float(e1 & 0xFFFF0000u);
+              f[4] += __uint_as_float(e2 << 16);
+              f[5] += __uint_as_float(e2 & 0xFFFF0000u);
+              f[6] += __uint_as_float(e3 << 16);
+              f[7] += __uint_as_float(e3 & 0xFFFF0000u);
+            }
+            const uint32_t o0 = pack_bf16(f[0], f[1]), o1 = pack_bf16(f[2], f[3]);
+            const uint32_t o2 = pack_bf16(f[4], f[5]), o3 = pack_bf16(f[6], f[7]);
+            asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};\n" ::"r"(addr), "r"(o0), "r"(o1), "r"(o2), "r"(o3)
+                         : "memory");
+          }
+          asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
+          __syncwarp();
+          if (lane == 0) {
+            if (rows_live) tma_store_3d(&maps.out, slab, q * kChunkCols + g * 64, s1, s2);
+            bulk_commit();
+            if (HAS_E) {
+              // the store before this one is done reading its stage: hand that stage back
+              bulk_wait_read<1>();
+              if (held >= 0) mbar_arrive(e_empty_bar(held));
+            }
+          }
+          held = eslot;
+        }
+      }
+    }
+    if (HAS_E && lane == 0) {
+      bulk_wait_read<0>();
+      if (held >= 0) mbar_arrive(e_empty_bar(held));
+    }
+    if (lane == 0) bulk_wait<0>();
+  }
+
+  asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
+  __syncthreads();
+  if (warp == 1) {
+    asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem_base),
+                 "r"(Cfg::kTmemCols) : "memory");
+  }
+}
+
+}  // namespace ssn
