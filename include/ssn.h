@@ -86,7 +86,26 @@ typedef struct ssn_codec {
   int64_t vocab;        /* rows of E (ignored when E is NULL)                             */
   const void *P;        /* device [max_pos x d] or NULL: no positional term (RoPE models) */
   int64_t ldp;          /* >= d                                                           */
+  /* Optional prepared tables (see ssn_prepare_tables), fp32, or NULL.  They are constants of
+   * the codec, like U, T_fixed and PE themselves, and only ssn_compress reads them.           */
+  const float *EU;      /* device [vocab x k] = E U, or NULL                              */
+  int64_t ldeu;         /* >= k                                                           */
+  const float *PU;      /* device [max_pos x k] = P U, or NULL                            */
+  int64_t ldpu;         /* >= k                                                           */
 } ssn_codec_t;
+
+/*
+ * Projects the codec's constant tables once: EU = E U [vocab x k] and PU = P U [max_pos x k],
+ * in fp32 (products of the stored values, fp32 accumulation).  Sec. 4.1 makes PE and T_fixed
+ * fixed and known to both ends, and U_k is fixed, so by linearity Eq. (ssn_compress) is
+ *     Z[t,:] = X[t,:] U - EU[ids[t],:] - PU[pos(t),:]
+ * and a codec whose EU / PU fields point at these tables lets ssn_compress read only X, ids
+ * and 2k floats per token instead of the E and P rows.  Either output may be NULL (then that
+ * table is not made; it must be NULL when the codec has no such term).  The tables must be
+ * made again whenever U, E or P change.  The codec passed in is read for U, E, P only.
+ */
+ssn_status_t ssn_prepare_tables(const ssn_codec_t *codec, float *EU, int64_t ldeu, float *PU,
+                                int64_t ldpu, void *stream);
 
 /*
  * Sender side, Eq. (ssn_compress):  Z[t,:] = (X[t,:] - P[pos(t),:] - E[ids[t],:]) U.

@@ -39,6 +39,8 @@ class ssn_codec_t(ctypes.Structure):
         ("U", ctypes.c_void_p), ("ldu", ctypes.c_int64),
         ("E", ctypes.c_void_p), ("lde", ctypes.c_int64), ("vocab", ctypes.c_int64),
         ("P", ctypes.c_void_p), ("ldp", ctypes.c_int64),
+        ("EU", ctypes.c_void_p), ("ldeu", ctypes.c_int64),
+        ("PU", ctypes.c_void_p), ("ldpu", ctypes.c_int64),
     ]
 
 
@@ -64,6 +66,7 @@ _SIGNATURES = {
     "ssn_weight_reproject": (_i32, [_codec_p, ctypes.POINTER(_vp), _i32, _i64, _i64, _i64, _i32,
                                     _vp, _sz, _vp]),
     "ssn_weight_reproject_left_static": (_i32, [_codec_p, _vp, _i64, _i64, _vp]),
+    "ssn_prepare_tables": (_i32, [_codec_p, _vp, _i64, _vp, _i64, _vp]),
     "ssn_static_scratch_bytes": (_sz, []),
     "ssn_status_string": (ctypes.c_char_p, [_i32]),
     "ssn_version": (_i32, []),
@@ -158,6 +161,13 @@ def ssn_weight_reproject_left_static(codec: ssn_codec_t, W: int, cols: int, ldw:
     k * cols * 4 exceeds ssn_static_scratch_bytes()."""
     _check(_lib.ssn_weight_reproject_left_static(ctypes.byref(codec), W or None, cols, ldw,
                                                  stream or None), "ssn_weight_reproject_left_static")
+
+
+def ssn_prepare_tables(codec: ssn_codec_t, EU: int, ldeu: int, PU: int, ldpu: int,
+                       stream: int = 0) -> None:
+    """EU [vocab x k] = E U and PU [max_pos x k] = P U in fp32 (0 = do not make that table)."""
+    _check(_lib.ssn_prepare_tables(ctypes.byref(codec), EU or None, ldeu, PU or None, ldpu,
+                                   stream or None), "ssn_prepare_tables")
 
 
 def raw(name: str):

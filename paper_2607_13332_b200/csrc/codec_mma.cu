@@ -221,11 +221,15 @@ cudaError_t launch_codec_umma_project(const MmaArgs &a, bool shift, int sm_count
   if (a.zout == nullptr || a.dst != nullptr || a.src == nullptr) return cudaErrorNotSupported;
   if (a.d % kUmmaCols != 0 || a.k > 128 || a.n < 4 * kUmmaTile || a.n > 0x7fffffffLL)
     return cudaErrorNotSupported;
-  const bool has_e = shift && a.shift.E != nullptr, has_p = shift && a.shift.P != nullptr;
+  // a term with a prepared table is subtracted in the epilogue and needs no operand
+  const bool has_e = shift && a.shift.E != nullptr && a.shift.EU == nullptr;
+  const bool has_p = shift && a.shift.P != nullptr && a.shift.PU == nullptr;
   if (has_p && (a.shift.pos != nullptr || a.shift.seq_len % kUmmaTile != 0 ||
                 a.shift.seq_len > a.shift.max_pos))
     return cudaErrorNotSupported;
   const int ntp = 2 * ((a.k + 15) / 16);
+  MmaArgs b = a;
+  if (!shift) b.shift.EU = b.shift.PU = nullptr;
   UmmaMaps maps;
   if (!make_sw128_map(&maps.x, a.src, a.n, a.d, a.lds, kUmmaTile)) return cudaErrorNotSupported;
   if (!make_sw128_map(&maps.u, a.U, a.d, a.k, a.ldu, kUmmaCols)) return cudaErrorNotSupported;
@@ -234,12 +238,12 @@ cudaError_t launch_codec_umma_project(const MmaArgs &a, bool shift, int sm_count
   maps.p = maps.x;
   if (has_p && !make_sw128_map(&maps.p, a.shift.P, a.shift.max_pos, a.d, a.shift.ldp, kUmmaTile))
     return cudaErrorNotSupported;
-  if (ntp <= 2) return launch_umma_ntp<2>(a, has_e, has_p, maps, sm_count, stream);
-  if (ntp <= 4) return launch_umma_ntp<4>(a, has_e, has_p, maps, sm_count, stream);
-  if (ntp <= 6) return launch_umma_ntp<6>(a, has_e, has_p, maps, sm_count, stream);
-  if (ntp <= 8) return launch_umma_ntp<8>(a, has_e, has_p, maps, sm_count, stream);
-  if (ntp <= 12) return launch_umma_ntp<12>(a, has_e, has_p, maps, sm_count, stream);
-  return launch_umma_ntp<16>(a, has_e, has_p, maps, sm_count, stream);
+  if (ntp <= 2) return launch_umma_ntp<2>(b, has_e, has_p, maps, sm_count, stream);
+  if (ntp <= 4) return launch_umma_ntp<4>(b, has_e, has_p, maps, sm_count, stream);
+  if (ntp <= 6) return launch_umma_ntp<6>(b, has_e, has_p, maps, sm_count, stream);
+  if (ntp <= 8) return launch_umma_ntp<8>(b, has_e, has_p, maps, sm_count, stream);
+  if (ntp <= 12) return launch_umma_ntp<12>(b, has_e, has_p, maps, sm_count, stream);
+  return launch_umma_ntp<16>(b, has_e, has_p, maps, sm_count, stream);
 }
 
 namespace {

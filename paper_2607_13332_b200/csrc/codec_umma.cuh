@@ -342,6 +342,23 @@ codec_umma_project_kernel(const MmaArgs a, const __grid_constant__ UmmaMaps maps
 
       const int64_t t = tile * kUmmaTile + quarter * 32 + lane;
       if (t < a.n) {
+        // terms that come from the prepared tables E U and P U (fp32) instead of an operand
+        auto subtract_row = [&](const float *row) {
+#pragma unroll
+          for (int q = 0; q < Cfg::kN / 16; ++q)
+#pragma unroll
+            for (int i = 0; i < 16; ++i)
+              if (q * 16 + i < a.k)
+                v[q][i] = __float_as_uint(__uint_as_float(v[q][i]) - __ldg(row + q * 16 + i));
+        };
+        if (!HAS_E && a.shift.EU != nullptr) {
+          const int64_t er = embedding_row(a.shift, t);
+          if (er >= 0) subtract_row(a.shift.EU + er * a.shift.ldeu);
+        }
+        if (!HAS_P && a.shift.PU != nullptr) {
+          const int64_t pr = position_row(a.shift, t);
+          if (pr >= 0) subtract_row(a.shift.PU + pr * a.shift.ldpu);
+        }
         __nv_bfloat16 *zrow = a.zout + t * a.ldzout;
 #pragma unroll
         for (int q = 0; q < Cfg::kN / 16; ++q) {

@@ -93,6 +93,47 @@ token_kernel(const TokenArgs a) {
   }
 }
 
+// ---- prepared tables: out [n x k] (fp32) = rows_in [n x d] U --------------------------------
+struct TableArgs {
+  const void *rows_in;   // E or P
+  const void *U;
+  float *out;
+  int64_t ld_in, ldu, ld_out, n;
+  int32_t d, k;
+};
+
+constexpr int kTableWarps = 8;
+
+// One warp per row; the lanes split d and reduce with shuffles, 8 columns of U at a time.
+template <typename T>
+__global__ void __launch_bounds__(kTableWarps * 32) table_project_kernel(const TableArgs a) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int64_t t = (int64_t)blockIdx.x * kTableWarps + warp;
+  if (t >= a.n) return;
+  const T *row = static_cast<const T *>(a.rows_in) + t * a.ld_in;
+  const T *U = static_cast<const T *>(a.U);
+  for (int j0 = 0; j0 < a.k; j0 += kGenericKChunk) {
+    const int jn = min(kGenericKChunk, a.k - j0);
+    float acc[kGenericKChunk];
+#pragma unroll
+    for (int jj = 0; jj < kGenericKChunk; ++jj) acc[jj] = 0.f;
+    for (int i = lane; i < a.d; i += 32) {
+      const float r = to_f32(row[i]);
+      const T *urow = U + (int64_t)i * a.ldu + j0;
+#pragma unroll
+      for (int jj = 0; jj < kGenericKChunk; ++jj)
+        if (jj < jn) acc[jj] = fmaf(r, to_f32(urow[jj]), acc[jj]);
+    }
+#pragma unroll
+    for (int jj = 0; jj < kGenericKChunk; ++jj) {
+      float v = acc[jj];
+#pragma unroll
+      for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
+      if (lane == 0 && jj < jn) a.out[t * a.ld_out + j0 + jj] = v;
+    }
+  }
+}
+
 // ---- LEFT re-projection, W [d x m]:  T = U^T W  then  W = U T ------------------------------
 struct LeftArgs {
   void *W;          // [d x m]

@@ -164,7 +164,52 @@ ssn_status_t ssn_compress(const ssn_codec_t *codec, const void *X, int64_t ldx,
   a.d = codec->d;
   a.k = codec->k;
   a.sub_shift = 1;
+  // prepared tables: only kernels that know them read them, the others use E and P
+  if (codec->E != nullptr && codec->EU != nullptr) {
+    if (codec->ldeu < codec->k) return SSN_ERR_SHAPE;
+    a.shift.EU = codec->EU;
+    a.shift.ldeu = codec->ldeu;
+  }
+  if (codec->P != nullptr && codec->PU != nullptr) {
+    if (codec->ldpu < codec->k) return SSN_ERR_SHAPE;
+    a.shift.PU = codec->PU;
+    a.shift.ldpu = codec->ldpu;
+  }
   return launch_token_kernel(a, codec->dtype, static_cast<cudaStream_t>(stream));
+}
+
+ssn_status_t ssn_prepare_tables(const ssn_codec_t *codec, float *EU, int64_t ldeu, float *PU,
+                                int64_t ldpu, void *stream) {
+  ssn_status_t st = check_codec(codec);
+  if (st != SSN_OK) return st;
+  if ((EU != nullptr && codec->E == nullptr) || (PU != nullptr && codec->P == nullptr)) return SSN_ERR_NULL;
+  if ((EU != nullptr && (ldeu < codec->k || codec->lde < codec->d || codec->vocab < 1)) ||
+      (PU != nullptr && (ldpu < codec->k || codec->ldp < codec->d || codec->max_pos < 1)))
+    return SSN_ERR_SHAPE;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  for (int which = 0; which < 2; ++which) {
+    float *out = which == 0 ? EU : PU;
+    if (out == nullptr) continue;
+    TableArgs t{};
+    t.rows_in = which == 0 ? codec->E : codec->P;
+    t.ld_in = which == 0 ? codec->lde : codec->ldp;
+    t.n = which == 0 ? codec->vocab : (int64_t)codec->max_pos;
+    t.U = codec->U;
+    t.ldu = codec->ldu;
+    t.out = out;
+    t.ld_out = which == 0 ? ldeu : ldpu;
+    t.d = codec->d;
+    t.k = codec->k;
+    const int64_t blocks = (t.n + kTableWarps - 1) / kTableWarps;
+    if (blocks > 0x7fffffffLL) return SSN_ERR_SHAPE;
+    if (codec->dtype == SSN_F32)
+      table_project_kernel<float><<<(unsigned)blocks, kTableWarps * 32, 0, s>>>(t);
+    else
+      table_project_kernel<__nv_bfloat16><<<(unsigned)blocks, kTableWarps * 32, 0, s>>>(t);
+    st = launch_status();
+    if (st != SSN_OK) return st;
+  }
+  return SSN_OK;
 }
 
 ssn_status_t ssn_decompress(const ssn_codec_t *codec, const void *Z, int64_t ldz,

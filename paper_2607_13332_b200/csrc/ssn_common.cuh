@@ -30,6 +30,9 @@ struct ShiftTables {
   int64_t lde, ldp, vocab;
   int32_t max_pos, seq_len;
   int32_t *dev_status; // nullable
+  const float *EU;     // [vocab x k] = E U in fp32, or nullptr (compress only)
+  const float *PU;     // [max_pos x k] = P U in fp32, or nullptr (compress only)
+  int64_t ldeu, ldpu;
 };
 
 // Row index into E for token t, or -1 for "no row" (table absent or id out of range, the

@@ -55,6 +55,7 @@ class Codec:
         for t in (U, E, P):
             if t is not None and (not t.is_cuda or t.dtype != _TORCH_DTYPE[dtype]):
                 raise ValueError("codec tensors must be CUDA tensors of the codec dtype")
+        self.EU = self.PU = None
         self.dev_status = torch.zeros(1, dtype=torch.int32, device=U.device)
         self.c = binding.make_codec(
             self.d, self.k, binding.DTYPES[dtype], U.data_ptr(), _ld(U),
@@ -62,6 +63,26 @@ class Codec:
             E.shape[0] if E is not None else 0,
             P.data_ptr() if P is not None else 0, _ld(P) if P is not None else None,
             P.shape[0] if P is not None else 0)
+
+    def prepare_tables(self) -> None:
+        """Project the codec's constant tables once (EU = E U, PU = P U, fp32) and attach them,
+        so that compress reads 2k floats per token instead of the E and P rows.  Call it again
+        after changing U, E or P in place."""
+        dev = self.U.device
+        self.EU = torch.empty((self.E.shape[0], self.k), dtype=torch.float32, device=dev) \
+            if self.E is not None else None
+        self.PU = torch.empty((self.P.shape[0], self.k), dtype=torch.float32, device=dev) \
+            if self.P is not None else None
+        binding.ssn_prepare_tables(self.c, self.EU.data_ptr() if self.EU is not None else 0, self.k,
+                                   self.PU.data_ptr() if self.PU is not None else 0, self.k, _stream())
+        if self.EU is not None:
+            self.c.EU, self.c.ldeu = self.EU.data_ptr(), self.k
+        if self.PU is not None:
+            self.c.PU, self.c.ldpu = self.PU.data_ptr(), self.k
+
+    def drop_tables(self) -> None:
+        self.c.EU = self.c.PU = None
+        self.EU = self.PU = None
 
     def _empty(self, rows: int, cols: int) -> torch.Tensor:
         return torch.empty((rows, cols), dtype=_TORCH_DTYPE[self.dtype], device=self.U.device)

@@ -1,0 +1,147 @@
+"""GPU parity for the shapes that reach the tcgen05 kernels (large token counts, d a multiple of
+128, k <= 64 for the expansion kernels) and for the prepared tables EU = E U, PU = P U, each
+against the CPU oracle element by element."""
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import ssn_oracle as oracle
+from paper_2607_13332_b200 import binding, synth
+from tests.harness import Codec, assert_close, f64, guards_intact, host64, padded, to_device
+
+pytestmark = pytest.mark.gpu
+
+# batch, seq_len, d, k, vocab: batches of 8 whole sequences whose length is a multiple of 16
+# take the 8 x 16 tiles of the expansion kernel, the others its 128-token tiles or the
+# mma.sync kernel
+SHAPES = [
+    (8, 128, 256, 40, 300),
+    (32, 256, 1024, 40, 5000),
+    (32, 64, 512, 16, 100),
+    (256, 16, 384, 64, 100),
+    (64, 48, 256, 33, 100),
+    (8, 80, 128, 8, 50),
+    (5, 200, 512, 40, 77),       # batch not a multiple of 8
+    (3, 333, 256, 24, 77),       # sequence length not a multiple of 16
+    (16, 64, 192, 40, 60),       # d not a multiple of 128
+    (16, 64, 256, 72, 60),       # k > 64
+]
+
+
+def _inputs(batch, seq_len, d, k, vocab, seed):
+    wl = synth.Workload("tc", d, k, vocab, batch, seq_len, synth.BF16)
+    t = synth.codec_inputs(wl, seed=seed, noise_std=1e-3)
+    return wl, t
+
+
+@pytest.mark.parametrize("batch,seq_len,d,k,vocab", SHAPES)
+@pytest.mark.parametrize("tables", ["EP", "E", "P", "none"])
+def test_decompress_and_compress_on_sequence_batches(batch, seq_len, d, k, vocab, tables):
+    wl, t = _inputs(batch, seq_len, d, k, vocab, seed=batch * 131 + seq_len + d + k)
+    dt, n = wl.dtype, wl.n_tokens
+    E0 = t["E"] if "E" in tables else None
+    P0 = t["P"] if "P" in tables else None
+    codec = Codec(dt, to_device(t["U"], dt), to_device(E0, dt), to_device(P0, dt))
+    ids = torch.from_numpy(t["ids"]).cuda()
+    U, E, P = f64(t["U"], dt), f64(E0, dt), f64(P0, dt)
+    pos = oracle.token_positions(n, seq_len)
+
+    Xh = codec.decompress(to_device(t["Z0"], dt), ids, seq_len=seq_len)
+    Xo, _ = oracle.decompress(f64(t["Z0"], dt), U, E, t["ids"], P, pos)
+    assert_close(host64(Xh, dt), Xo, dt, "decompress")
+
+    X = to_device(t["X"], dt)
+    Zo, _ = oracle.compress(f64(t["X"], dt), U, E, t["ids"], P, pos)
+    assert_close(host64(codec.compress(X, ids, seq_len=seq_len), dt), Zo, dt, "compress")
+    if tables != "none":
+        codec.prepare_tables()
+        assert_close(host64(codec.compress(X, ids, seq_len=seq_len), dt), Zo, dt, "compress, prepared tables")
+    assert codec.take_status() == 0
+
+
+def test_prepared_tables_match_their_definition():
+    for dt in (synth.F32, synth.BF16):
+        wl = synth.Workload("tab", 384, 24, 211, 2, 96, dt)
+        t = synth.codec_inputs(wl, seed=77)
+        codec = Codec(dt, to_device(t["U"], dt), to_device(t["E"], dt), to_device(t["P"], dt))
+        codec.prepare_tables()
+        U, E, P = f64(t["U"], dt), f64(t["E"], dt), f64(t["P"], dt)
+        for got, src in ((codec.EU, E), (codec.PU, P)):
+            want = src @ U
+            err = np.abs(got.double().cpu().numpy() - want).max() / np.abs(want).max()
+            assert err < 2e-6, err
+
+
+def test_prepared_tables_with_explicit_positions_and_bad_indices():
+    """Explicit positions, a ragged token count, ids and positions out of range: the table path
+    drops the same terms and raises the same status bits as the row path."""
+    wl, t = _inputs(1, 1000, 512, 40, 90, seed=5)
+    dt, n = wl.dtype, wl.n_tokens
+    rng = np.random.default_rng(3)
+    ids_np = t["ids"].copy()
+    pos_np = rng.integers(0, wl.seq_len, n).astype(np.int32)
+    ids_np[[3, 500]] = [-1, wl.vocab]
+    pos_np[[7, 999]] = [wl.seq_len, -5]
+    codec = Codec(dt, to_device(t["U"], dt), to_device(t["E"], dt), to_device(t["P"], dt))
+    ids, pos = torch.from_numpy(ids_np).cuda(), torch.from_numpy(pos_np).cuda()
+    X = to_device(t["X"], dt)
+    Zo, flags = oracle.compress(f64(t["X"], dt), f64(t["U"], dt), f64(t["E"], dt), ids_np,
+                                f64(t["P"], dt), pos_np)
+    Z_rows = codec.compress(X, ids, pos=pos)
+    status_rows = codec.take_status()
+    codec.prepare_tables()
+    Z_tab = codec.compress(X, ids, pos=pos)
+    status_tab = codec.take_status()
+    assert_close(host64(Z_rows, dt), Zo, dt, "rows")
+    assert_close(host64(Z_tab, dt), Zo, dt, "tables")
+    assert status_rows == status_tab == (binding.SSN_DEV_BAD_ID | binding.SSN_DEV_BAD_POS) == flags
+
+
+def test_prepare_tables_argument_errors():
+    wl, t = _inputs(1, 64, 128, 8, 20, seed=1)
+    dt = wl.dtype
+    codec = Codec(dt, to_device(t["U"], dt))
+    out = torch.empty((64, 8), dtype=torch.float32, device="cuda")
+    fn = binding.raw("ssn_prepare_tables")
+    assert fn(codec.c, out.data_ptr(), 8, None, 8, None) == binding.SSN_ERR_NULL      # no E in the codec
+    codec2 = Codec(dt, to_device(t["U"], dt), to_device(t["E"], dt))
+    assert fn(codec2.c, out.data_ptr(), 4, None, 8, None) == binding.SSN_ERR_SHAPE    # ldeu < k
+    assert fn(codec2.c, None, 8, None, 8, None) == binding.SSN_OK                     # nothing to make
+
+
+@pytest.mark.parametrize("rows,d,k", [(512, 256, 40), (1000, 512, 8), (2125, 1024, 64), (640, 384, 33),
+                                      (3000, 2048, 16), (4096, 4096, 40)])
+def test_project_then_expand_in_place_with_guard_bands(rows, d, k):
+    """Weight re-projection (in place) and the projected gradient (out of place, with the
+    coordinates) at sizes that take the fused tcgen05 kernel; nothing outside the rows moves."""
+    dt = synth.BF16
+    U0 = synth.to_storage(synth.subspace_basis(d, k, seed=rows + k), dt)
+    W0 = synth.to_storage(np.random.default_rng(rows).standard_normal((rows, d)) * 0.05, dt)
+    codec = Codec(dt, to_device(U0, dt))
+    U, Wf = f64(U0, dt), f64(W0, dt)
+    view, buf = padded(rows, d, d + 64, dt, fill=to_device(W0, dt))
+    codec.weight_reproject([view], "right")
+    assert_close(host64(view, dt), oracle.weight_reproject(Wf, U, "right"), dt, "reproject right")
+    assert guards_intact(view, buf, dt)
+
+    G = to_device(W0, dt)
+    dZ, Gp = codec.grad_project(G, full=True)
+    assert_close(host64(Gp, dt), oracle.grad_project_full(Wf, U), dt, "grad full")
+    assert_close(host64(dZ, dt), oracle.grad_project_coeff(Wf, U), dt, "grad coeff")
+    assert torch.equal(G, to_device(W0, dt))     # the input is not touched
+
+
+def test_decompress_output_guard_bands_and_leading_dimensions():
+    wl, t = _inputs(8, 64, 256, 40, 50, seed=9)
+    dt, n = wl.dtype, wl.n_tokens
+    codec = Codec(dt, to_device(t["U"], dt), to_device(t["E"], dt), to_device(t["P"], dt))
+    ids = torch.from_numpy(t["ids"]).cuda()
+    Zin, _ = padded(n, wl.k, wl.k + 24, dt, fill=to_device(t["Z0"], dt))
+    out, buf = padded(n, wl.d, wl.d + 128, dt)
+    codec.decompress(Zin, ids, seq_len=wl.seq_len, out=out)
+    Xo, _ = oracle.decompress(f64(t["Z0"], dt), f64(t["U"], dt), f64(t["E"], dt), t["ids"],
+                              f64(t["P"], dt), oracle.token_positions(n, wl.seq_len))
+    assert_close(host64(out, dt), Xo, dt, "decompress into a padded view")
+    assert guards_intact(out, buf, dt)
+    assert codec.take_status() == 0
