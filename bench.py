@@ -272,16 +272,13 @@ def run_ours(args):
     Z_h, dZ_h = Z.cpu().pin_memory(), dZ.cpu().pin_memory()
     weights = [to_device(synth.projection_weight(r, c, 0x5EED, dt, layer=i), dt)
                for i, (r, c) in enumerate(synth.REPROJECT_SHAPES_8B.values())]
-    groups = [[w] for w in weights]
-    work = [codec.reproject_workspace(w.shape[0], w.shape[1], "right", 1) for w in weights]
     del t["X"], t["G"], t["E"]
 
     stream = torch.cuda.current_stream()
     kernel_events = []
 
-    def reproject():
-        for g, ws in zip(groups, work):
-            codec.weight_reproject(g, "right", workspace=ws)
+    def reproject():     # both projections of the block in one call (and one launch)
+        codec.weight_reproject_rows(weights)
 
     calls = (("compress", lambda: codec.compress(X, ids, seq_len=wl.seq_len, out=Z)),
              ("decompress", lambda: codec.decompress(Z, ids, seq_len=wl.seq_len, out=Xh)),

@@ -167,6 +167,18 @@ ssn_status_t ssn_weight_reproject(const ssn_codec_t *codec, void *const *W_ptrs,
                                   void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * The RIGHT re-projection W_i <- (W_i U) U^T of `count` weights [rows[i] x d] that may differ in
+ * their number of rows (all output projections of a block after one optimizer step, Sec. 4.1),
+ * in place, with as few launches as possible.
+ *   W_ptrs, rows, ldw   HOST arrays of `count` device pointers, row counts (>= 1) and leading
+ *                       dimensions (>= d); the weights must be distinct buffers.
+ * Same arithmetic as ssn_weight_reproject(..., SSN_SIDE_RIGHT, ...); needs no workspace.
+ */
+ssn_status_t ssn_weight_reproject_rows(const ssn_codec_t *codec, void *const *W_ptrs,
+                                       const int64_t *rows, const int64_t *ldw, int32_t count,
+                                       void *stream);
+
+/*
  * LEFT re-projection of ONE weight, W [d x cols] <- U (U^T W), without a caller workspace.
  * (The paper has no counterpart: this is a packaging variant of ssn_weight_reproject.)
  *

@@ -257,30 +257,60 @@ cudaError_t launch_roundtrip_ntp(const MmaArgs &a, const UmmaRoundTripMaps &maps
     if (e != cudaSuccess) return e;
     configured = true;
   }
-  int64_t grid = (a.n + kUmmaTile - 1) / kUmmaTile;
+  int64_t grid = maps.tile_start[maps.count];
   if (grid > sm_count) grid = sm_count;
   kernel<<<(unsigned)grid, kRoundTripThreads, smem, stream>>>(a, maps);
   return cudaGetLastError();
 }
 }  // namespace
 
-// Project-then-expand on tcgen05 (weight re-projection, projected gradient).  Returns
-// cudaErrorNotSupported when the call should take the mma.sync kernels instead: k > 64, d not
-// a multiple of 128, few rows, no tensor map (unaligned base or leading dimension).
-cudaError_t launch_codec_umma_roundtrip(const MmaArgs &a, int sm_count, cudaStream_t stream) {
-  if (a.src == nullptr || a.dst == nullptr) return cudaErrorNotSupported;
-  if (a.d % kChunkCols != 0 || a.k > 64 || a.n < 4 * kUmmaTile || a.n > 0x7fffffffLL)
-    return cudaErrorNotSupported;
+// Project-then-expand on tcgen05 for `count` matrices [rows[i] x d] at once (src[i] -> dst[i], which
+// may be the same buffer).  Returns cudaErrorNotSupported when the call should take the mma.sync
+// kernels instead: k > 64, d not a multiple of 128, few rows in all, too many matrices, no tensor map
+// (unaligned base or leading dimension).  zout (coordinates, bf16) only with one matrix.
+cudaError_t launch_codec_umma_roundtrip_list(const MmaArgs &a, const __nv_bfloat16 *const *src,
+                                             __nv_bfloat16 *const *dst, const int64_t *rows,
+                                             const int64_t *lds, const int64_t *lddst, int count,
+                                             int sm_count, cudaStream_t stream) {
+  if (count < 1 || count > kRoundTripMaxMatrices) return cudaErrorNotSupported;
+  if (a.d % kChunkCols != 0 || a.k > 64) return cudaErrorNotSupported;
   UmmaRoundTripMaps maps;
-  if (!make_sw128_map(&maps.s, a.src, a.n, a.d, a.lds, kUmmaTile)) return cudaErrorNotSupported;
+  int64_t tiles = 0, total = 0;
+  for (int i = 0; i < count; ++i) {
+    if (src[i] == nullptr || dst[i] == nullptr || rows[i] < 1 || rows[i] > 0x7fffffffLL) return cudaErrorNotSupported;
+    maps.tile_start[i] = (int32_t)tiles;
+    maps.rows[i] = rows[i];
+    tiles += (rows[i] + kUmmaTile - 1) / kUmmaTile;
+    total += rows[i];
+    if (tiles > 0x3fffffffLL) return cudaErrorNotSupported;
+    if (!make_sw128_map(&maps.s[i], src[i], rows[i], a.d, lds[i], kUmmaTile)) return cudaErrorNotSupported;
+    if (!make_sw128_map(&maps.out[i], dst[i], rows[i], a.d, lddst[i], 32)) return cudaErrorNotSupported;
+  }
+  if (total < 4 * kUmmaTile) return cudaErrorNotSupported;
+  for (int i = count; i < kRoundTripMaxMatrices; ++i) {
+    maps.s[i] = maps.s[0];
+    maps.out[i] = maps.out[0];
+    maps.rows[i] = 0;
+    maps.tile_start[i + 1] = (int32_t)tiles;
+  }
+  maps.tile_start[count] = (int32_t)tiles;
+  maps.count = count;
   if (!make_sw128_map(&maps.u, a.U, a.d, a.k, a.ldu, kUmmaCols)) return cudaErrorNotSupported;
   if (!make_sw128_map(&maps.u_wide, a.U, a.d, 64, a.ldu, kUmmaCols)) return cudaErrorNotSupported;
-  if (!make_sw128_map(&maps.out, a.dst, a.n, a.d, a.lddst, 32)) return cudaErrorNotSupported;
+  MmaArgs b = a;
+  if (count > 1) b.zout = nullptr;
   const int ntp = 2 * ((a.k + 15) / 16);
-  if (ntp <= 2) return launch_roundtrip_ntp<2>(a, maps, sm_count, stream);
-  if (ntp <= 4) return launch_roundtrip_ntp<4>(a, maps, sm_count, stream);
-  if (ntp <= 6) return launch_roundtrip_ntp<6>(a, maps, sm_count, stream);
-  return launch_roundtrip_ntp<8>(a, maps, sm_count, stream);
+  if (ntp <= 2) return launch_roundtrip_ntp<2>(b, maps, sm_count, stream);
+  if (ntp <= 4) return launch_roundtrip_ntp<4>(b, maps, sm_count, stream);
+  if (ntp <= 6) return launch_roundtrip_ntp<6>(b, maps, sm_count, stream);
+  return launch_roundtrip_ntp<8>(b, maps, sm_count, stream);
+}
+
+cudaError_t launch_codec_umma_roundtrip(const MmaArgs &a, int sm_count, cudaStream_t stream) {
+  if (a.src == nullptr || a.dst == nullptr || a.n > 0x7fffffffLL) return cudaErrorNotSupported;
+  const __nv_bfloat16 *src = a.src;
+  __nv_bfloat16 *dst = a.dst;
+  return launch_codec_umma_roundtrip_list(a, &src, &dst, &a.n, &a.lds, &a.lddst, 1, sm_count, stream);
 }
 
 // Expansion (decompress) on tcgen05.  Returns cudaErrorNotSupported when the call should take the

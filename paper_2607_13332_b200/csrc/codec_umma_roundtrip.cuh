@@ -72,9 +72,18 @@ struct UmmaRoundTripConfig {
   static constexpr int kSmemBytes = 1024 + kStagesN * kStageBytes + kFixedBytes + kBars * 8 + 16;
 };
 
+constexpr int kRoundTripMaxMatrices = 8;
+
+// One launch takes up to kRoundTripMaxMatrices matrices [rows_i x d] (the output projections of
+// a block, say): the tiles of all of them are dealt to the CTAs as one list.
 struct UmmaRoundTripMaps {
-  // S: boxes of 128 rows x 64 cols; U: 64 x 64 (u_wide: see UmmaMaps); out: 32 rows x 64 cols
-  CUtensorMap s, u, u_wide, out;
+  // U: 64 x 64 boxes (u_wide: see UmmaMaps); per matrix, S: boxes of 128 rows x 64 columns,
+  // out: 32 rows x 64 columns
+  CUtensorMap u, u_wide;
+  CUtensorMap s[kRoundTripMaxMatrices], out[kRoundTripMaxMatrices];
+  int64_t rows[kRoundTripMaxMatrices];
+  int32_t tile_start[kRoundTripMaxMatrices + 1];   // first tile of each matrix; [count] = all tiles
+  int32_t count;
 };
 
 template <int NTP>
@@ -86,7 +95,13 @@ codec_umma_roundtrip_kernel(const MmaArgs a, const __grid_constant__ UmmaRoundTr
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int nstage = a.d / kUmmaCols;
   const int nchunks = a.d / kChunkCols;
-  const int64_t ntiles = (a.n + kUmmaTile - 1) / kUmmaTile;
+  const int64_t ntiles = maps.tile_start[maps.count];
+  // tile -> matrix and first row
+  auto locate = [&](int64_t tile, int &w, int &row0) {
+    w = 0;
+    while (w + 1 < maps.count && tile >= maps.tile_start[w + 1]) ++w;
+    row0 = (int)(tile - maps.tile_start[w]) * kUmmaTile;
+  };
 
   const uint32_t smem0 = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t c_hi = smem0, c_lo = smem0 + Cfg::kTileBytes;
@@ -143,13 +158,14 @@ codec_umma_roundtrip_kernel(const MmaArgs a, const __grid_constant__ UmmaRoundTr
     int slot = 0;
     uint32_t parity = 1;   // a fresh "empty" barrier passes a wait on parity 1
     for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
-      const int row0 = (int)(tile * kUmmaTile);
+      int w, row0;
+      locate(tile, w, row0);
       for (int st = 0; st < nstage; ++st) {
         if (!dead && !mbar_wait(empty_bar(slot), parity)) timed_out();
         const uint32_t base = ring + (uint32_t)slot * Cfg::kStageBytes;
         if (lane == 0) {
           mbar_expect_tx(full_bar(slot), Cfg::kStageBytes);
-          tma_load_2d(base, &maps.s, full_bar(slot), st * kUmmaCols, row0);
+          tma_load_2d(base, &maps.s[w], full_bar(slot), st * kUmmaCols, row0);
           tma_load_2d(base + Cfg::kTileBytes, st == nstage - 1 ? &maps.u : &maps.u_wide, full_bar(slot), 0,
                       st * kUmmaCols);
         }
@@ -242,7 +258,9 @@ codec_umma_roundtrip_kernel(const MmaArgs a, const __grid_constant__ UmmaRoundTr
     const bool zvec = a.zout != nullptr && ((a.ldzout & 7) == 0) && ((reinterpret_cast<uintptr_t>(a.zout) & 15) == 0);
     int64_t tcount = 0, ccount = 0;
     for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x, ++tcount) {
-      const int64_t row0 = tile * kUmmaTile;
+      int w, row0;
+      locate(tile, w, row0);
+      const int64_t nrows = maps.rows[w];
       // ---- split: C (fp32, TMEM) -> C_hi, C_lo (bf16, shared memory)
       if (!dead && !mbar_wait(acc1_full_bar, (uint32_t)(tcount & 1))) timed_out();
       asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
@@ -265,7 +283,7 @@ codec_umma_roundtrip_kernel(const MmaArgs a, const __grid_constant__ UmmaRoundTr
               hi[i] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
               lo[i] = pack_bf16(f0 - __bfloat162float(h0), f1 - __bfloat162float(h1));
             }
-            if (a.zout != nullptr && t < a.n) {
+            if (a.zout != nullptr && t < nrows) {
               __nv_bfloat16 *zrow = a.zout + t * a.ldzout;
               if (zvec && c * 8 + 8 <= a.k) {
                 *reinterpret_cast<uint4 *>(zrow + c * 8) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
@@ -324,8 +342,8 @@ codec_umma_roundtrip_kernel(const MmaArgs a, const __grid_constant__ UmmaRoundTr
           asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
           __syncwarp();
           if (lane == 0) {
-            if (row0 + quarter * 32 < a.n)
-              tma_store_2d(&maps.out, slab, q * kChunkCols + g * 64, (int)(row0 + quarter * 32));
+            if (row0 + quarter * 32 < nrows)
+              tma_store_2d(&maps.out[w], slab, q * kChunkCols + g * 64, (int)(row0 + quarter * 32));
             bulk_commit();
           }
         }

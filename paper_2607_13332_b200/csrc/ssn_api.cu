@@ -6,6 +6,7 @@
 #include <cuda_runtime.h>
 
 #include <atomic>
+#include <vector>
 
 #include "codec_mma_launch.h"
 #include "generic_kernels.cuh"
@@ -135,6 +136,59 @@ ssn_status_t launch_token_kernel(const TokenArgs &a, int32_t dtype, cudaStream_t
   return launch_status();
 }
 
+}  // namespace
+}  // namespace ssn
+
+namespace ssn {
+namespace {
+// RIGHT re-projection of `count` matrices [rows[i] x d]: groups of up to 8 go to the fused
+// tcgen05 kernel in one launch each; what that kernel does not take goes matrix by matrix.
+ssn_status_t reproject_right_list(const ssn_codec_t *codec, void *const *W_ptrs, const int64_t *rows,
+                                  const int64_t *ldw, int32_t count, cudaStream_t s) {
+  const int sms = sm_count_of_current_device();
+  int32_t done = 0;
+  while (done < count) {
+    const int32_t take = count - done < 8 ? count - done : 8;
+    bool fused = false;
+    if (codec->dtype == SSN_BF16 && sms > 0 && aligned16(codec->U) && (codec->ldu & 7) == 0) {
+      MmaArgs m{};
+      m.U = static_cast<const __nv_bfloat16 *>(codec->U);
+      m.ldu = codec->ldu;
+      m.d = codec->d;
+      m.k = codec->k;
+      const __nv_bfloat16 *src[8];
+      __nv_bfloat16 *dst[8];
+      for (int32_t i = 0; i < take; ++i) src[i] = dst[i] = static_cast<__nv_bfloat16 *>(W_ptrs[done + i]);
+      cudaError_t e = launch_codec_umma_roundtrip_list(m, src, dst, rows + done, ldw + done, ldw + done, take,
+                                                       sms, s);
+      if (e == cudaSuccess) {
+        g_launches.fetch_add(1, std::memory_order_relaxed);
+        fused = true;
+      } else if (e != cudaErrorNotSupported) {
+        return SSN_ERR_CUDA;
+      }
+    }
+    if (!fused) {
+      // Every row of W is one "token": project onto U and expand again, no shift terms.
+      for (int32_t b = done; b < done + take; ++b) {
+        TokenArgs a{};
+        a.src = W_ptrs[b];
+        a.lds = ldw[b];
+        a.dst = W_ptrs[b];
+        a.lddst = ldw[b];
+        a.U = codec->U;
+        a.ldu = codec->ldu;
+        a.n = rows[b];
+        a.d = codec->d;
+        a.k = codec->k;
+        ssn_status_t st = launch_token_kernel(a, codec->dtype, s);
+        if (st != SSN_OK) return st;
+      }
+    }
+    done += take;
+  }
+  return SSN_OK;
+}
 }  // namespace
 }  // namespace ssn
 
@@ -276,6 +330,20 @@ size_t ssn_weight_reproject_workspace_bytes(const ssn_codec_t *codec, int64_t ro
   return 0;
 }
 
+ssn_status_t ssn_weight_reproject_rows(const ssn_codec_t *codec, void *const *W_ptrs, const int64_t *rows,
+                                       const int64_t *ldw, int32_t count, void *stream) {
+  ssn_status_t st = check_codec(codec);
+  if (st != SSN_OK) return st;
+  if (count < 0) return SSN_ERR_SHAPE;
+  if (count == 0) return SSN_OK;
+  if (W_ptrs == nullptr || rows == nullptr || ldw == nullptr) return SSN_ERR_NULL;
+  for (int32_t b = 0; b < count; ++b) {
+    if (W_ptrs[b] == nullptr) return SSN_ERR_NULL;
+    if (rows[b] < 1 || ldw[b] < codec->d) return SSN_ERR_SHAPE;
+  }
+  return reproject_right_list(codec, W_ptrs, rows, ldw, count, static_cast<cudaStream_t>(stream));
+}
+
 ssn_status_t ssn_weight_reproject(const ssn_codec_t *codec, void *const *W_ptrs, int32_t batch,
                                   int64_t rows, int64_t cols, int64_t ldw, int32_t side,
                                   void *workspace, size_t workspace_bytes, void *stream) {
@@ -293,22 +361,8 @@ ssn_status_t ssn_weight_reproject(const ssn_codec_t *codec, void *const *W_ptrs,
   cudaStream_t s = static_cast<cudaStream_t>(stream);
 
   if (side == SSN_SIDE_RIGHT) {
-    // Every row of W is one "token": project onto U and expand again, no shift terms.
-    for (int32_t b = 0; b < batch; ++b) {
-      TokenArgs a{};
-      a.src = W_ptrs[b];
-      a.lds = ldw;
-      a.dst = W_ptrs[b];
-      a.lddst = ldw;
-      a.U = codec->U;
-      a.ldu = codec->ldu;
-      a.n = rows;
-      a.d = codec->d;
-      a.k = codec->k;
-      st = launch_token_kernel(a, codec->dtype, s);
-      if (st != SSN_OK) return st;
-    }
-    return SSN_OK;
+    std::vector<int64_t> nrows((size_t)batch, rows), lds((size_t)batch, ldw);
+    return reproject_right_list(codec, W_ptrs, nrows.data(), lds.data(), batch, s);
   }
 
   const int64_t col_blocks = (cols + kLeftCols - 1) / kLeftCols;

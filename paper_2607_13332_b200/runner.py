@@ -130,6 +130,13 @@ class Codec:
             return None
         return torch.empty(nbytes, dtype=torch.uint8, device=self.U.device)
 
+    def weight_reproject_rows(self, weights: Sequence[torch.Tensor]) -> None:
+        """In place, RIGHT side, for weights [rows_i x d] of any row counts."""
+        if weights:
+            binding.ssn_weight_reproject_rows(self.c, [w.data_ptr() for w in weights],
+                                              [w.shape[0] for w in weights], [_ld(w) for w in weights],
+                                              _stream())
+
     def weight_reproject(self, weights: Sequence[torch.Tensor], side: str,
                          workspace: Optional[torch.Tensor] = None) -> None:
         """In place, for a list of equally shaped weights."""

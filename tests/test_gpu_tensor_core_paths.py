@@ -145,3 +145,44 @@ def test_decompress_output_guard_bands_and_leading_dimensions():
     assert_close(host64(out, dt), Xo, dt, "decompress into a padded view")
     assert guards_intact(out, buf, dt)
     assert codec.take_status() == 0
+
+
+def test_reproject_rows_list_of_unequal_weights():
+    """Several weights with different row counts in one call (one launch of the fused kernel),
+    in place, against the oracle; then the shapes the fused kernel does not take."""
+    dt, d, k = synth.BF16, 512, 40
+    U0 = synth.to_storage(synth.subspace_basis(d, k, seed=3), dt)
+    codec = Codec(dt, to_device(U0, dt))
+    U = f64(U0, dt)
+    rows = [640, 130, 1, 1024, 77, 256, 300, 128, 999, 64]      # more than one launch's worth
+    W0s = [synth.to_storage(np.random.default_rng(r).standard_normal((r, d)) * 0.05, dt) for r in rows]
+    views = [padded(r, d, d + 8 * (i % 3), dt, fill=to_device(w, dt)) for i, (r, w) in enumerate(zip(rows, W0s))]
+    codec.weight_reproject_rows([v for v, _ in views])
+    for (v, buf), w0 in zip(views, W0s):
+        assert_close(host64(v, dt), oracle.weight_reproject(f64(w0, dt), U, "right"), dt, f"rows {v.shape[0]}")
+        assert guards_intact(v, buf, dt)
+    # fp32 and a rank above 64 take the general path, same results
+    for dt2, k2 in ((synth.F32, 24), (synth.BF16, 72)):
+        U2 = synth.to_storage(synth.subspace_basis(d, k2, seed=4), dt2)
+        c2 = Codec(dt2, to_device(U2, dt2))
+        Ws0 = [synth.to_storage(np.random.default_rng(r).standard_normal((r, d)) * 0.05, dt2) for r in (600, 50)]
+        Ws = [to_device(w, dt2) for w in Ws0]
+        c2.weight_reproject_rows(Ws)
+        for w, w0 in zip(Ws, Ws0):
+            assert_close(host64(w, dt2), oracle.weight_reproject(f64(w0, dt2), f64(U2, dt2), "right"), dt2, "general")
+
+
+def test_reproject_rows_argument_errors():
+    import ctypes
+    dt, d, k = synth.BF16, 256, 8
+    codec = Codec(dt, to_device(synth.to_storage(synth.subspace_basis(d, k, seed=3), dt), dt))
+    W = torch.zeros((16, d), dtype=torch.bfloat16, device="cuda")
+    fn = binding.raw("ssn_weight_reproject_rows")
+    ptrs, one = (ctypes.c_void_p * 1)(W.data_ptr()), ctypes.c_int64
+    assert fn(codec.c, ptrs, (one * 1)(16), (one * 1)(d), 1, None) == binding.SSN_OK
+    assert fn(codec.c, ptrs, (one * 1)(0), (one * 1)(d), 1, None) == binding.SSN_ERR_SHAPE
+    assert fn(codec.c, ptrs, (one * 1)(16), (one * 1)(d - 1), 1, None) == binding.SSN_ERR_SHAPE
+    assert fn(codec.c, None, (one * 1)(16), (one * 1)(d), 1, None) == binding.SSN_ERR_NULL
+    assert fn(codec.c, (ctypes.c_void_p * 1)(None), (one * 1)(16), (one * 1)(d), 1, None) == binding.SSN_ERR_NULL
+    assert fn(codec.c, ptrs, (one * 1)(16), (one * 1)(d), 0, None) == binding.SSN_OK
+    assert fn(codec.c, ptrs, (one * 1)(16), (one * 1)(d), -1, None) == binding.SSN_ERR_SHAPE
