@@ -182,7 +182,8 @@ cudaError_t launch_umma_expand_one(const MmaArgs &a, const ExpandGeometry &geo, 
     if (e != cudaSuccess) return e;
     configured = true;
   }
-  int64_t grid = geo.ntiles < sm_count ? geo.ntiles : sm_count;
+  const int64_t units = geo.ntiles * (a.d / kChunkCols);     // (tile, chunk) pairs, dealt evenly
+  int64_t grid = units < sm_count ? units : sm_count;
   kernel<<<(unsigned)grid, kExpandThreads, smem, stream>>>(a, geo, maps);
   return cudaGetLastError();
 }

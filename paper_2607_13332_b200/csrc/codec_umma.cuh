@@ -294,7 +294,7 @@ codec_umma_project_kernel(const MmaArgs a, const __grid_constant__ UmmaMaps maps
           if (!dead && !mbar_wait(empty_bar(slot), parity)) timed_out();
           const uint32_t base = smem0 + (uint32_t)slot * Cfg::kStageBytes;
 #pragma unroll
-          for (int i = 0; i < 8; ++i) cp_async16(base + dst[i], src[i] + st * 128, 16);
+          for (int i = 0; i < 8; ++i) cp_async16_cg(base + dst[i], src[i] + st * 128);
           cp_async_commit();
           if (++pending > Cfg::kGatherLag) {
             cp_async_wait<Cfg::kGatherLag>();

@@ -50,7 +50,7 @@ struct UmmaExpandConfig {
   static constexpr int kU2Bytes = kChunkCols * 128;             // 128 rows of U, K-major
   static constexpr int kPBytes = HAS_P ? 2 * kGridPos * 128 : 0;   // 16 rows of P, two 64-column groups
   static constexpr int kUStageBytes = kU2Bytes + kPBytes;
-  static constexpr int kUStages = 3;
+  static constexpr int kUStages = HAS_E ? 2 : 3;   // with E the shared memory is better spent on its ring
   static constexpr int kEStageBytes = kTileBytes;               // E rows of 64 columns of a chunk
   // Without E the epilogue warps stage their output in two [32 x 128 B] slabs each; with E the
   // sum is formed in place in the E stage, which is then the source of the TMA store.
@@ -159,6 +159,15 @@ codec_umma_expand_kernel(const MmaArgs a, const ExpandGeometry geo, const __grid
     dead = true;
     if (a.shift.dev_status) atomicOr(a.shift.dev_status, SSN_DEV_TIMEOUT);
   };
+  // Work is dealt in units of (tile, chunk): chunks are independent output columns, so a CTA takes
+  // a contiguous, balanced range of units and may start and end in the middle of a tile.
+  const int64_t units = ntiles * nchunks;
+  const int64_t u_lo = (units * blockIdx.x) / gridDim.x, u_hi = (units * (blockIdx.x + 1)) / gridDim.x;
+  const int64_t tile_lo = u_lo / nchunks, tile_hi = u_hi > u_lo ? (u_hi - 1) / nchunks : tile_lo - 1;
+  auto chunk_range = [&](int64_t tile, int &q0, int &q1) {
+    q0 = tile == tile_lo ? (int)(u_lo - tile_lo * nchunks) : 0;
+    q1 = tile == tile_hi ? (int)(u_hi - tile_hi * nchunks) : nchunks;
+  };
   // tile -> TMA coordinates (row coordinate, sequence coordinate) of its first token
   auto tile_coords = [&](int64_t tile, int &c1, int &c2) {
     if (geo.grid_mode) {
@@ -176,7 +185,7 @@ codec_umma_expand_kernel(const MmaArgs a, const ExpandGeometry geo, const __grid
     int slot = 0;
     uint32_t parity = 1;
     int64_t tcount = 0;
-    for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x, ++tcount) {
+    for (int64_t tile = tile_lo; tile <= tile_hi; ++tile, ++tcount) {
       int c1, c2;
       tile_coords(tile, c1, c2);
       const int zb = (int)(tcount & 1);
@@ -185,7 +194,9 @@ codec_umma_expand_kernel(const MmaArgs a, const ExpandGeometry geo, const __grid
         mbar_expect_tx(z_full_bar(zb), Cfg::kTileBytes);
         tma_load_3d(z_base + zb * Cfg::kTileBytes, &maps.z, z_full_bar(zb), 0, c1, c2);
       }
-      for (int q = 0; q < nchunks; ++q) {
+      int q0, q1;
+      chunk_range(tile, q0, q1);
+      for (int q = q0; q < q1; ++q) {
         if (!dead && !mbar_wait(u_empty_bar(slot), parity)) timed_out();
         const uint32_t base = u_ring + (uint32_t)slot * Cfg::kUStageBytes;
         if (lane == 0) {
@@ -216,11 +227,13 @@ codec_umma_expand_kernel(const MmaArgs a, const ExpandGeometry geo, const __grid
       int slot = 0;
       uint32_t parity = 0;
       int64_t tcount = 0, ccount = 0;
-      for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x, ++tcount) {
+      for (int64_t tile = tile_lo; tile <= tile_hi; ++tile, ++tcount) {
         const int zb = (int)(tcount & 1);
         if (!dead && !mbar_wait(z_full_bar(zb), (uint32_t)((tcount >> 1) & 1))) timed_out();
         const uint64_t zd = kdesc + ((z_base + zb * Cfg::kTileBytes) >> 4);
-        for (int q = 0; q < nchunks; ++q, ++ccount) {
+        int q0, q1;
+        chunk_range(tile, q0, q1);
+        for (int q = q0; q < q1; ++q, ++ccount) {
           const int db = (int)(ccount & 1);
           if (!dead && !mbar_wait(d_empty_bar(db), (uint32_t)(((ccount >> 1) & 1) ^ 1))) timed_out();
           if (!dead && !mbar_wait(u_full_bar(slot), parity)) timed_out();
@@ -232,7 +245,7 @@ codec_umma_expand_kernel(const MmaArgs a, const ExpandGeometry geo, const __grid
           if (HAS_P) umma_bf16(dacc, seld, pdesc + ((base + Cfg::kU2Bytes) >> 4), idesc_kmn, 1u);
           umma_commit(u_empty_bar(slot));
           umma_commit(d_full_bar(db));
-          if (q == nchunks - 1) umma_commit(z_empty_bar(zb));
+          if (q == q1 - 1) umma_commit(z_empty_bar(zb));
           if (++slot == SU) {
             slot = 0;
             parity ^= 1u;
@@ -250,7 +263,7 @@ codec_umma_expand_kernel(const MmaArgs a, const ExpandGeometry geo, const __grid
       const int piece = lane & 7, sub = lane >> 3;
       int slot = 0;
       uint32_t parity = 1;
-      for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+      for (int64_t tile = tile_lo; tile <= tile_hi; ++tile) {
         int c1, c2;
         tile_coords(tile, c1, c2);
         const unsigned char *src[8];
@@ -266,11 +279,13 @@ codec_umma_expand_kernel(const MmaArgs a, const ExpandGeometry geo, const __grid
                             : g_zero_row) + piece * 16;
           dst[i] = r * 128 + ((piece ^ (r & 7)) << 4);
         }
-        for (int qg = 0; qg < 2 * nchunks; ++qg) {     // 64-column groups of the row
+        int q0, q1;
+        chunk_range(tile, q0, q1);
+        for (int qg = 2 * q0; qg < 2 * q1; ++qg) {     // 64-column groups of the row
           if (!dead && !mbar_wait(e_empty_bar(slot), parity)) timed_out();
           const uint32_t base = e_ring + (uint32_t)slot * Cfg::kEStageBytes;
 #pragma unroll
-          for (int i = 0; i < 8; ++i) cp_async16(base + dst[i], src[i] + qg * 128, 16);
+          for (int i = 0; i < 8; ++i) cp_async16_cg(base + dst[i], src[i] + qg * 128);
           asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];\n" ::"r"(e_full_bar(slot)) : "memory");
           if (++slot == SE) {
             slot = 0;
@@ -289,14 +304,16 @@ codec_umma_expand_kernel(const MmaArgs a, const ExpandGeometry geo, const __grid
     const uint32_t slab0 = staging + (uint32_t)(group * 4 + quarter) * 8192;   // !HAS_E: two slabs
     int64_t ccount = 0;
     int held = -1;                                // E stage whose store may still be reading it
-    for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+    for (int64_t tile = tile_lo; tile <= tile_hi; ++tile) {
       int c1, c2;
       tile_coords(tile, c1, c2);
       // first token row of this warp's 32 rows, as TMA store coordinates
       const int s1 = geo.grid_mode ? c1 : c1 + quarter * 32;
       const int s2 = geo.grid_mode ? c2 + quarter * (32 / kGridPos) : 0;
       const bool rows_live = geo.grid_mode || (int64_t)s1 < a.n;
-      for (int q = 0; q < nchunks; ++q, ++ccount) {
+      int q0, q1;
+      chunk_range(tile, q0, q1);
+      for (int q = q0; q < q1; ++q, ++ccount) {
         if ((int)(ccount & 1) != group) continue;
         const int db = group;
         if (!dead && !mbar_wait(d_full_bar(db), (uint32_t)((ccount >> 1) & 1))) timed_out();
