@@ -61,6 +61,9 @@ def parse_args():
                          "the E and P rows (the default step gathers; the table variant is always "
                          "timed beside it as compress_prepared_tables)")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
+    ap.add_argument("--sweep", choices=["compress", "reproject"], default=None,
+                    help="instead of the step: time the compress sweep (d, k, tokens) or the "
+                         "re-projection sweep (k, weight shape, 32 layers); one JSON line per point")
     return ap.parse_args()
 
 
@@ -392,8 +395,87 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def run_sweep(args):
+    """Benchmark definition's sweeps, one GPU: device-resident inputs larger than L2 where the
+    point allows, CUDA events around `reps` back-to-back launches after 3 warm-up launches."""
+    import torch
+
+    import __graft_entry__ as entry
+    entry.build()
+    from paper_2607_13332_b200 import synth
+    from paper_2607_13332_b200.runner import Codec, to_device
+
+    peak, _ = measured_hbm_peak()
+    dt, vocab, seq = synth.BF16, 128256, 2048
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(1)
+
+    def timed_us(fn, reps):
+        for _ in range(3):
+            fn()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        a.record()
+        for _ in range(reps):
+            fn()
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) * 1e3 / reps
+
+    if args.sweep == "compress":
+        for d in (1024, 2048, 4096, 8192):
+            E = (torch.randn((vocab, d), device="cuda", generator=gen) * 0.02).bfloat16()
+            P = to_device(synth.to_storage(synth.sinusoidal_positions(seq, d), dt), dt)
+            for k in (8, 32, 64, 128):
+                U = to_device(synth.to_storage(synth.subspace_basis(d, k, 1), dt), dt)
+                codec, codec_t = Codec(dt, U, E, P), Codec(dt, U, E, P)
+                codec_t.prepare_tables()
+                for n in (4096, 65536, 524288):
+                    ids_np = np.random.default_rng(n + d + k).integers(0, vocab, n).astype(np.int32)
+                    ids = torch.from_numpy(ids_np).cuda()
+                    X = torch.randn((n, d), device="cuda", generator=gen).bfloat16()
+                    Z = torch.empty((n, k), dtype=torch.bfloat16, device="cuda")
+                    uniq = int(np.unique(ids_np).size)
+                    reps = 20 if n <= 65536 else 5
+                    out = {"sweep": "compress", "d": d, "k": k, "tokens": n, "distinct_ids": uniq}
+                    for name, c, algo in (
+                            ("rows", codec, n * d * 2 + uniq * d * 2 + min(seq, n) * d * 2 + d * k * 2 + n * k * 2),
+                            ("tables", codec_t, n * d * 2 + n * 4 + (uniq + min(seq, n)) * k * 4 + d * k * 2 + n * k * 2)):
+                        us = timed_us(lambda: c.compress(X, ids, seq_len=seq, out=Z), reps)
+                        out[name] = {"us": round(us, 1), "GBps": round(algo / us / 1e3, 0),
+                                     "frac_of_measured": round(algo / us / 1e3 / peak, 3)}
+                    status = codec.take_status() | codec_t.take_status()
+                    out["status"] = status
+                    print(json.dumps(out), flush=True)
+                    del X, Z, ids
+            del E, P
+    else:
+        d = 4096
+        for k in synth.REPROJECT_RANKS:
+            U = to_device(synth.to_storage(synth.subspace_basis(d, k, 1), dt), dt)
+            codec = Codec(dt, U)
+            for name, (rows, cols) in synth.REPROJECT_SHAPES_8B.items():
+                Ws = [(torch.randn((rows, cols), device="cuda", generator=gen) * 0.02).bfloat16()
+                      for _ in range(32)]
+                algo = 32 * 2 * rows * cols * 2
+                us = timed_us(lambda: codec.weight_reproject_rows(Ws), 5)
+                out = {"sweep": "reproject", "k": k, "weight": name, "shape": [rows, cols], "layers": 32,
+                       "right": {"us": round(us, 1), "GBps": round(algo / us / 1e3, 0),
+                                 "frac_of_measured": round(algo / us / 1e3 / peak, 3)}}
+                if rows == cols:
+                    ws = codec.reproject_workspace(rows, cols, "left", 32)
+                    us = timed_us(lambda: codec.weight_reproject(Ws, "left", workspace=ws), 3)
+                    out["left"] = {"us": round(us, 1), "GBps": round(algo / us / 1e3, 0),
+                                   "frac_of_measured": round(algo / us / 1e3 / peak, 3)}
+                print(json.dumps(out), flush=True)
+                del Ws
+
+
 def main():
     args = parse_args()
+    if args.sweep is not None:
+        run_sweep(args)
+        return
     if args.impl == "reference":
         run_reference(args)
     else:

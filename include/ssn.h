@@ -167,15 +167,23 @@ ssn_status_t ssn_weight_reproject(const ssn_codec_t *codec, void *const *W_ptrs,
                                   void *workspace, size_t workspace_bytes, void *stream);
 
 /*
- * The RIGHT re-projection W_i <- (W_i U) U^T of `count` weights [rows[i] x d] that may differ in
- * their number of rows (all output projections of a block after one optimizer step, Sec. 4.1),
- * in place, with as few launches as possible.
- *   W_ptrs, rows, ldw   HOST arrays of `count` device pointers, row counts (>= 1) and leading
- *                       dimensions (>= d); the weights must be distinct buffers.
- * Same arithmetic as ssn_weight_reproject(..., SSN_SIDE_RIGHT, ...); needs no workspace.
+ * The re-projection of `count` weights that may differ in their free extent (all output
+ * projections of a block after one optimizer step, Sec. 4.1), in place, with as few launches as
+ * possible:
+ *   SSN_SIDE_RIGHT: W_i is [extent[i] x d],  W_i <- (W_i U) U^T
+ *   SSN_SIDE_LEFT : W_i is [d x extent[i]],  W_i <- U (U^T W_i)
+ *   W_ptrs, extent, ldw   HOST arrays of `count` device pointers, extents (>= 1) and leading
+ *                         dimensions (>= d for RIGHT, >= extent[i] for LEFT); distinct buffers.
+ *   workspace   only read for SSN_SIDE_LEFT weights that the fused tensor-core kernel does not
+ *               take (fp32, k > 64, d not a multiple of 128, leading dimension not a multiple of
+ *               8 elements, unaligned base): k * max(extent) * 4 bytes, 16-byte aligned; such a
+ *               weight without enough workspace gives SSN_ERR_WORKSPACE (weights before it in the
+ *               list have been re-projected then).  May be NULL otherwise.
+ * Same arithmetic as ssn_weight_reproject.
  */
-ssn_status_t ssn_weight_reproject_rows(const ssn_codec_t *codec, void *const *W_ptrs,
-                                       const int64_t *rows, const int64_t *ldw, int32_t count,
+ssn_status_t ssn_weight_reproject_list(const ssn_codec_t *codec, void *const *W_ptrs,
+                                       const int64_t *extent, const int64_t *ldw, int32_t count,
+                                       int32_t side, void *workspace, size_t workspace_bytes,
                                        void *stream);
 
 /*
@@ -198,7 +206,9 @@ ssn_status_t ssn_weight_reproject_rows(const ssn_codec_t *codec, void *const *W_
  *   Sharing: every call on a device uses the same array.  Its contents are rewritten completely
  *          by each call, so nothing has to be cleared, but two calls that overlap on the GPU
  *          (different streams, no ordering between them) race on it: order them.
- * Same arithmetic and results as ssn_weight_reproject(..., SSN_SIDE_LEFT, ...) on one weight.
+ * Same arithmetic and results as the general (workspace) form of ssn_weight_reproject(...,
+ * SSN_SIDE_LEFT, ...) on one weight; the fused tensor-core form of that call needs no scratch
+ * at all and differs from this one only in rounding order.
  */
 #define SSN_STATIC_SCRATCH_BYTES (4u << 20)
 ssn_status_t ssn_weight_reproject_left_static(const ssn_codec_t *codec, void *W, int64_t cols,

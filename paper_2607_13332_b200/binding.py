@@ -67,8 +67,8 @@ _SIGNATURES = {
                                     _vp, _sz, _vp]),
     "ssn_weight_reproject_left_static": (_i32, [_codec_p, _vp, _i64, _i64, _vp]),
     "ssn_prepare_tables": (_i32, [_codec_p, _vp, _i64, _vp, _i64, _vp]),
-    "ssn_weight_reproject_rows": (_i32, [_codec_p, ctypes.POINTER(_vp), ctypes.POINTER(_i64),
-                                         ctypes.POINTER(_i64), _i32, _vp]),
+    "ssn_weight_reproject_list": (_i32, [_codec_p, ctypes.POINTER(_vp), ctypes.POINTER(_i64),
+                                         ctypes.POINTER(_i64), _i32, _i32, _vp, _sz, _vp]),
     "ssn_static_scratch_bytes": (_sz, []),
     "ssn_status_string": (ctypes.c_char_p, [_i32]),
     "ssn_version": (_i32, []),
@@ -165,11 +165,13 @@ def ssn_weight_reproject_left_static(codec: ssn_codec_t, W: int, cols: int, ldw:
                                                  stream or None), "ssn_weight_reproject_left_static")
 
 
-def ssn_weight_reproject_rows(codec: ssn_codec_t, W_ptrs, rows, ldw, stream: int = 0) -> None:
-    """RIGHT re-projection of weights [rows[i] x d] with different row counts, in place."""
+def ssn_weight_reproject_list(codec: ssn_codec_t, W_ptrs, extent, ldw, side: int, workspace: int = 0,
+                              workspace_bytes: int = 0, stream: int = 0) -> None:
+    """Re-projection of weights [extent[i] x d] (RIGHT) or [d x extent[i]] (LEFT), in place."""
     n = len(W_ptrs)
-    _check(_lib.ssn_weight_reproject_rows(ctypes.byref(codec), (_vp * n)(*W_ptrs), (_i64 * n)(*rows),
-                                          (_i64 * n)(*ldw), n, stream or None), "ssn_weight_reproject_rows")
+    _check(_lib.ssn_weight_reproject_list(ctypes.byref(codec), (_vp * n)(*W_ptrs), (_i64 * n)(*extent),
+                                          (_i64 * n)(*ldw), n, side, workspace or None, workspace_bytes,
+                                          stream or None), "ssn_weight_reproject_list")
 
 
 def ssn_prepare_tables(codec: ssn_codec_t, EU: int, ldeu: int, PU: int, ldpu: int,

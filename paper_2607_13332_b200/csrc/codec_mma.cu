@@ -248,9 +248,9 @@ cudaError_t launch_codec_umma_project(const MmaArgs &a, bool shift, int sm_count
 }
 
 namespace {
-template <int NTP>
+template <int NTP, bool LEFT>
 cudaError_t launch_roundtrip_ntp(const MmaArgs &a, const UmmaRoundTripMaps &maps, int sm_count, cudaStream_t stream) {
-  auto kernel = codec_umma_roundtrip_kernel<NTP>;
+  auto kernel = codec_umma_roundtrip_kernel<NTP, LEFT>;
   constexpr int smem = UmmaRoundTripConfig<NTP>::kSmemBytes;
   static bool configured = false;
   if (!configured) {
@@ -272,7 +272,7 @@ cudaError_t launch_roundtrip_ntp(const MmaArgs &a, const UmmaRoundTripMaps &maps
 cudaError_t launch_codec_umma_roundtrip_list(const MmaArgs &a, const __nv_bfloat16 *const *src,
                                              __nv_bfloat16 *const *dst, const int64_t *rows,
                                              const int64_t *lds, const int64_t *lddst, int count,
-                                             int sm_count, cudaStream_t stream) {
+                                             int sm_count, cudaStream_t stream, bool left) {
   if (count < 1 || count > kRoundTripMaxMatrices) return cudaErrorNotSupported;
   if (a.d % kChunkCols != 0 || a.k > 64) return cudaErrorNotSupported;
   UmmaRoundTripMaps maps;
@@ -284,8 +284,13 @@ cudaError_t launch_codec_umma_roundtrip_list(const MmaArgs &a, const __nv_bfloat
     tiles += (rows[i] + kUmmaTile - 1) / kUmmaTile;
     total += rows[i];
     if (tiles > 0x3fffffffLL) return cudaErrorNotSupported;
-    if (!make_sw128_map(&maps.s[i], src[i], rows[i], a.d, lds[i], kUmmaTile)) return cudaErrorNotSupported;
-    if (!make_sw128_map(&maps.out[i], dst[i], rows[i], a.d, lddst[i], 32)) return cudaErrorNotSupported;
+    if (left) {   // [d x rows[i]]: `rows` counts the columns, which are what a tile spans
+      if (!make_sw128_map(&maps.s[i], src[i], a.d, rows[i], lds[i], kUmmaCols)) return cudaErrorNotSupported;
+      if (!make_sw128_map(&maps.out[i], dst[i], a.d, rows[i], lddst[i], 32)) return cudaErrorNotSupported;
+    } else {
+      if (!make_sw128_map(&maps.s[i], src[i], rows[i], a.d, lds[i], kUmmaTile)) return cudaErrorNotSupported;
+      if (!make_sw128_map(&maps.out[i], dst[i], rows[i], a.d, lddst[i], 32)) return cudaErrorNotSupported;
+    }
   }
   if (total < 4 * kUmmaTile) return cudaErrorNotSupported;
   for (int i = count; i < kRoundTripMaxMatrices; ++i) {
@@ -299,19 +304,25 @@ cudaError_t launch_codec_umma_roundtrip_list(const MmaArgs &a, const __nv_bfloat
   if (!make_sw128_map(&maps.u, a.U, a.d, a.k, a.ldu, kUmmaCols)) return cudaErrorNotSupported;
   if (!make_sw128_map(&maps.u_wide, a.U, a.d, 64, a.ldu, kUmmaCols)) return cudaErrorNotSupported;
   MmaArgs b = a;
-  if (count > 1) b.zout = nullptr;
+  if (count > 1 || left) b.zout = nullptr;
   const int ntp = 2 * ((a.k + 15) / 16);
-  if (ntp <= 2) return launch_roundtrip_ntp<2>(b, maps, sm_count, stream);
-  if (ntp <= 4) return launch_roundtrip_ntp<4>(b, maps, sm_count, stream);
-  if (ntp <= 6) return launch_roundtrip_ntp<6>(b, maps, sm_count, stream);
-  return launch_roundtrip_ntp<8>(b, maps, sm_count, stream);
+  if (left) {
+    if (ntp <= 2) return launch_roundtrip_ntp<2, true>(b, maps, sm_count, stream);
+    if (ntp <= 4) return launch_roundtrip_ntp<4, true>(b, maps, sm_count, stream);
+    if (ntp <= 6) return launch_roundtrip_ntp<6, true>(b, maps, sm_count, stream);
+    return launch_roundtrip_ntp<8, true>(b, maps, sm_count, stream);
+  }
+  if (ntp <= 2) return launch_roundtrip_ntp<2, false>(b, maps, sm_count, stream);
+  if (ntp <= 4) return launch_roundtrip_ntp<4, false>(b, maps, sm_count, stream);
+  if (ntp <= 6) return launch_roundtrip_ntp<6, false>(b, maps, sm_count, stream);
+  return launch_roundtrip_ntp<8, false>(b, maps, sm_count, stream);
 }
 
 cudaError_t launch_codec_umma_roundtrip(const MmaArgs &a, int sm_count, cudaStream_t stream) {
   if (a.src == nullptr || a.dst == nullptr || a.n > 0x7fffffffLL) return cudaErrorNotSupported;
   const __nv_bfloat16 *src = a.src;
   __nv_bfloat16 *dst = a.dst;
-  return launch_codec_umma_roundtrip_list(a, &src, &dst, &a.n, &a.lds, &a.lddst, 1, sm_count, stream);
+  return launch_codec_umma_roundtrip_list(a, &src, &dst, &a.n, &a.lds, &a.lddst, 1, sm_count, stream, false);
 }
 
 // Expansion (decompress) on tcgen05.  Returns cudaErrorNotSupported when the call should take the

@@ -23,13 +23,14 @@ struct MmaArgs {
 // Shapes the tensor-core kernels take (alignment is checked by the caller).
 bool codec_mma_supports(int d, int k);
 
-// Project-then-expand of up to 8 matrices [rows[i] x d] in ONE launch of the tcgen05 kernel
-// (a.U, a.ldu, a.d, a.k are read from `a`); cudaErrorNotSupported when the shapes or
+// Project-then-expand of up to 8 matrices in ONE launch of the tcgen05 kernel (a.U, a.ldu, a.d,
+// a.k are read from `a`): [rows[i] x d] with the subspace on the columns, or, with `left`,
+// [d x rows[i]] with the subspace on the rows.  cudaErrorNotSupported when the shapes or
 // alignments are not the kernel's, and nothing has been launched then.
 cudaError_t launch_codec_umma_roundtrip_list(const MmaArgs &a, const __nv_bfloat16 *const *src,
                                              __nv_bfloat16 *const *dst, const int64_t *rows,
                                              const int64_t *lds, const int64_t *lddst, int count,
-                                             int sm_count, cudaStream_t stream);
+                                             int sm_count, cudaStream_t stream, bool left);
 
 // mode: 1 = project, 2 = expand, 3 = project then expand (shift must be false).
 cudaError_t launch_codec_mma(const MmaArgs &a, bool shift, int mode, int sm_count,

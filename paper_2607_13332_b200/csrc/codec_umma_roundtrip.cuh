@@ -20,8 +20,14 @@
 //   warp 0  pass-1 producer     warp 1  MMA issuer, owns the TMEM allocation
 //   warps 2-5  epilogue (TMEM lanes 32*(warp%4) ..)     warp 6  pass-2 producer (U chunks)
 //
-// Rows of a tile are only written after all of them have been read, and tiles are disjoint, so
-// the call may be in place.  Every wait is bounded; a wait that runs out sets SSN_DEV_TIMEOUT
+// LEFT variant (W stored [d x m], the subspace on the rows: W <- U (U^T W)): a tile is a block of
+// 128 COLUMNS of W over all d rows.  Pass 1 contracts over the rows, T^T = W_blk^T U, with the block
+// as an MN-major A operand (boxes of 64 rows x 64 columns, as stored); pass 2 swaps the roles,
+// D[128 rows x 128 columns] = U_chunk (A, K-major) x (C_hi + C_lo) (B, K-major), and the epilogue
+// stores rows of W as before.
+//
+// Rows (columns) of a tile are only written after all of them have been read, and tiles are
+// disjoint, so the call may be in place.  Every wait is bounded; a wait that runs out sets SSN_DEV_TIMEOUT
 // (when the caller gave a status word) and the kernel still runs to its end.
 #pragma once
 
@@ -86,7 +92,7 @@ struct UmmaRoundTripMaps {
   int32_t count;
 };
 
-template <int NTP>
+template <int NTP, bool LEFT>
 __global__ void __launch_bounds__(kRoundTripThreads, 1)
 codec_umma_roundtrip_kernel(const MmaArgs a, const __grid_constant__ UmmaRoundTripMaps maps) {
   using Cfg = UmmaRoundTripConfig<NTP>;
@@ -96,7 +102,7 @@ codec_umma_roundtrip_kernel(const MmaArgs a, const __grid_constant__ UmmaRoundTr
   const int nstage = a.d / kUmmaCols;
   const int nchunks = a.d / kChunkCols;
   const int64_t ntiles = maps.tile_start[maps.count];
-  // tile -> matrix and first row
+  // tile -> matrix and first row (LEFT: first column)
   auto locate = [&](int64_t tile, int &w, int &row0) {
     w = 0;
     while (w + 1 < maps.count && tile >= maps.tile_start[w + 1]) ++w;
@@ -165,7 +171,12 @@ codec_umma_roundtrip_kernel(const MmaArgs a, const __grid_constant__ UmmaRoundTr
         const uint32_t base = ring + (uint32_t)slot * Cfg::kStageBytes;
         if (lane == 0) {
           mbar_expect_tx(full_bar(slot), Cfg::kStageBytes);
-          tma_load_2d(base, &maps.s[w], full_bar(slot), st * kUmmaCols, row0);
+          if (LEFT) {   // rows st*64.. of the column block: two boxes of 64 columns
+            tma_load_2d(base, &maps.s[w], full_bar(slot), row0, st * kUmmaCols);
+            tma_load_2d(base + Cfg::kTileBytes / 2, &maps.s[w], full_bar(slot), row0 + 64, st * kUmmaCols);
+          } else {
+            tma_load_2d(base, &maps.s[w], full_bar(slot), st * kUmmaCols, row0);
+          }
           tma_load_2d(base + Cfg::kTileBytes, st == nstage - 1 ? &maps.u : &maps.u_wide, full_bar(slot), 0,
                       st * kUmmaCols);
         }
@@ -200,11 +211,13 @@ codec_umma_roundtrip_kernel(const MmaArgs a, const __grid_constant__ UmmaRoundTr
   } else if (warp == 1) {
     // ------------------------------------------------------------------------- MMA issuer
     if (lane == 0) {
-      constexpr uint32_t idesc1 = umma_idesc(Cfg::kN, false);
+      // LEFT: the A operand of pass 1 is MN-major as well (bit 15)
+      constexpr uint32_t idesc1 = umma_idesc(Cfg::kN, false) | (LEFT ? (1u << 15) : 0u);
       constexpr uint32_t idesc2 = umma_idesc_kk(kChunkCols);
       // descriptors without the start address, which is added per instruction (address / 16)
       const uint64_t kdesc = umma_desc(0, 16, 1024, 2);                 // K-major tile, rows of 128 B
       const uint64_t udesc = umma_desc(0, Cfg::kUBytes, 1024, 2);       // U slice of pass 1 (MN-major)
+      const uint64_t wdesc = umma_desc(0, Cfg::kTileBytes / 2, 1024, 2);  // LEFT: W block, two 64-column groups
       int slot = 0, uslot = 0;
       uint32_t parity = 0, uparity = 0;
       int64_t tcount = 0, ccount = 0;
@@ -214,10 +227,10 @@ codec_umma_roundtrip_kernel(const MmaArgs a, const __grid_constant__ UmmaRoundTr
           if (!dead && !mbar_wait(full_bar(slot), parity)) timed_out();
           asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
           const uint32_t base = ring + (uint32_t)slot * Cfg::kStageBytes;
-          const uint64_t ad = kdesc + (base >> 4), bd = udesc + ((base + Cfg::kTileBytes) >> 4);
+          const uint64_t ad = (LEFT ? wdesc : kdesc) + (base >> 4), bd = udesc + ((base + Cfg::kTileBytes) >> 4);
 #pragma unroll
-          for (int j = 0; j < kUmmaCols / 16; ++j)
-            umma_bf16(acc1, ad + j * 2, bd + j * 128, idesc1, (st > 0 || j > 0) ? 1u : 0u);
+          for (int j = 0; j < kUmmaCols / 16; ++j)   // a K step: 32 bytes of a K-major row, 16 rows of an MN-major tile
+            umma_bf16(acc1, ad + j * (LEFT ? 128 : 2), bd + j * 128, idesc1, (st > 0 || j > 0) ? 1u : 0u);
           umma_commit(empty_bar(slot));
           if (++slot == S) {
             slot = 0;
@@ -237,8 +250,13 @@ codec_umma_roundtrip_kernel(const MmaArgs a, const __grid_constant__ UmmaRoundTr
           const uint64_t hd = kdesc + (c_hi >> 4), ld = kdesc + (c_lo >> 4);
 #pragma unroll
           for (int j = 0; j < Cfg::kKSteps; ++j) {
-            umma_bf16(dacc, hd + j * 2, bd + j * 2, idesc2, j > 0 ? 1u : 0u);
-            umma_bf16(dacc, ld + j * 2, bd + j * 2, idesc2, 1u);
+            if (LEFT) {   // rows of U times the coordinates of the column block
+              umma_bf16(dacc, bd + j * 2, hd + j * 2, idesc2, j > 0 ? 1u : 0u);
+              umma_bf16(dacc, bd + j * 2, ld + j * 2, idesc2, 1u);
+            } else {
+              umma_bf16(dacc, hd + j * 2, bd + j * 2, idesc2, j > 0 ? 1u : 0u);
+              umma_bf16(dacc, ld + j * 2, bd + j * 2, idesc2, 1u);
+            }
           }
           umma_commit(u2_empty_bar(uslot));
           umma_commit(d_full_bar(db));
@@ -283,7 +301,7 @@ codec_umma_roundtrip_kernel(const MmaArgs a, const __grid_constant__ UmmaRoundTr
               hi[i] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
               lo[i] = pack_bf16(f0 - __bfloat162float(h0), f1 - __bfloat162float(h1));
             }
-            if (a.zout != nullptr && t < nrows) {
+            if (!LEFT && a.zout != nullptr && t < nrows) {
               __nv_bfloat16 *zrow = a.zout + t * a.ldzout;
               if (zvec && c * 8 + 8 <= a.k) {
                 *reinterpret_cast<uint4 *>(zrow + c * 8) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
@@ -342,8 +360,12 @@ codec_umma_roundtrip_kernel(const MmaArgs a, const __grid_constant__ UmmaRoundTr
           asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
           __syncwarp();
           if (lane == 0) {
-            if (row0 + quarter * 32 < nrows)
+            if (LEFT) {   // rows q*128 + 32*quarter .. of W, columns of this block
+              if (row0 + g * 64 < nrows)
+                tma_store_2d(&maps.out[w], slab, row0 + g * 64, q * kChunkCols + quarter * 32);
+            } else if (row0 + quarter * 32 < nrows) {
               tma_store_2d(&maps.out[w], slab, q * kChunkCols + g * 64, (int)(row0 + quarter * 32));
+            }
             bulk_commit();
           }
         }

@@ -160,7 +160,7 @@ ssn_status_t reproject_right_list(const ssn_codec_t *codec, void *const *W_ptrs,
       __nv_bfloat16 *dst[8];
       for (int32_t i = 0; i < take; ++i) src[i] = dst[i] = static_cast<__nv_bfloat16 *>(W_ptrs[done + i]);
       cudaError_t e = launch_codec_umma_roundtrip_list(m, src, dst, rows + done, ldw + done, ldw + done, take,
-                                                       sms, s);
+                                                       sms, s, false);
       if (e == cudaSuccess) {
         g_launches.fetch_add(1, std::memory_order_relaxed);
         fused = true;
@@ -182,6 +182,84 @@ ssn_status_t reproject_right_list(const ssn_codec_t *codec, void *const *W_ptrs,
         a.d = codec->d;
         a.k = codec->k;
         ssn_status_t st = launch_token_kernel(a, codec->dtype, s);
+        if (st != SSN_OK) return st;
+      }
+    }
+    done += take;
+  }
+  return SSN_OK;
+}
+}  // namespace
+}  // namespace ssn
+
+namespace ssn {
+namespace {
+// LEFT re-projection of up to 8 weights [d x cols[i]] on the fused tcgen05 kernel; false when
+// that kernel does not take the call (nothing launched).
+bool try_reproject_left_fused(const ssn_codec_t *codec, void *const *W_ptrs, const int64_t *cols,
+                              const int64_t *ldw, int32_t count, cudaStream_t s, ssn_status_t *st) {
+  *st = SSN_OK;
+  const int sms = sm_count_of_current_device();
+  if (codec->dtype != SSN_BF16 || sms <= 0 || !aligned16(codec->U) || (codec->ldu & 7) != 0) return false;
+  MmaArgs m{};
+  m.U = static_cast<const __nv_bfloat16 *>(codec->U);
+  m.ldu = codec->ldu;
+  m.d = codec->d;
+  m.k = codec->k;
+  const __nv_bfloat16 *src[8];
+  __nv_bfloat16 *dst[8];
+  for (int32_t i = 0; i < count; ++i) src[i] = dst[i] = static_cast<__nv_bfloat16 *>(W_ptrs[i]);
+  cudaError_t e = launch_codec_umma_roundtrip_list(m, src, dst, cols, ldw, ldw, count, sms, s, true);
+  if (e == cudaErrorNotSupported) return false;
+  if (e == cudaSuccess)
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+  else
+    *st = SSN_ERR_CUDA;
+  return true;
+}
+
+// LEFT re-projection of one weight with the general two-kernel form (T = U^T W in the workspace).
+ssn_status_t reproject_left_general(const ssn_codec_t *codec, void *W, int64_t cols, int64_t ldw,
+                                    void *workspace, size_t workspace_bytes, cudaStream_t s) {
+  if (workspace == nullptr || workspace_bytes < (size_t)codec->k * (size_t)cols * sizeof(float))
+    return SSN_ERR_WORKSPACE;
+  const int64_t col_blocks = (cols + kLeftCols - 1) / kLeftCols;
+  if (col_blocks > 0x7fffffffLL) return SSN_ERR_SHAPE;
+  LeftArgs a{};
+  a.W = W;
+  a.U = codec->U;
+  a.T = static_cast<float *>(workspace);
+  a.ldw = ldw;
+  a.ldu = codec->ldu;
+  a.m = cols;
+  a.d = codec->d;
+  a.k = codec->k;
+  dim3 g1((unsigned)col_blocks, (unsigned)((codec->k + kGenericKChunk - 1) / kGenericKChunk));
+  dim3 g2((unsigned)col_blocks, (unsigned)((codec->d + 31) / 32));
+  if (codec->dtype == SSN_F32) {
+    left_reduce_kernel<float><<<g1, kLeftCols, 0, s>>>(a);
+    left_expand_kernel<float><<<g2, kLeftCols, 0, s>>>(a);
+  } else {
+    left_reduce_kernel<__nv_bfloat16><<<g1, kLeftCols, 0, s>>>(a);
+    left_expand_kernel<__nv_bfloat16><<<g2, kLeftCols, 0, s>>>(a);
+  }
+  return launch_status(2);
+}
+
+// LEFT re-projection of `count` weights [d x cols[i]]: groups of up to 8 on the fused kernel, the
+// rest one by one through the workspace.
+ssn_status_t reproject_left_list(const ssn_codec_t *codec, void *const *W_ptrs, const int64_t *cols,
+                                 const int64_t *ldw, int32_t count, void *workspace,
+                                 size_t workspace_bytes, cudaStream_t s) {
+  int32_t done = 0;
+  while (done < count) {
+    const int32_t take = count - done < 8 ? count - done : 8;
+    ssn_status_t st;
+    if (try_reproject_left_fused(codec, W_ptrs + done, cols + done, ldw + done, take, s, &st)) {
+      if (st != SSN_OK) return st;
+    } else {
+      for (int32_t b = done; b < done + take; ++b) {
+        st = reproject_left_general(codec, W_ptrs[b], cols[b], ldw[b], workspace, workspace_bytes, s);
         if (st != SSN_OK) return st;
       }
     }
@@ -330,18 +408,23 @@ size_t ssn_weight_reproject_workspace_bytes(const ssn_codec_t *codec, int64_t ro
   return 0;
 }
 
-ssn_status_t ssn_weight_reproject_rows(const ssn_codec_t *codec, void *const *W_ptrs, const int64_t *rows,
-                                       const int64_t *ldw, int32_t count, void *stream) {
+ssn_status_t ssn_weight_reproject_list(const ssn_codec_t *codec, void *const *W_ptrs,
+                                       const int64_t *extent, const int64_t *ldw, int32_t count,
+                                       int32_t side, void *workspace, size_t workspace_bytes,
+                                       void *stream) {
   ssn_status_t st = check_codec(codec);
   if (st != SSN_OK) return st;
+  if (side != SSN_SIDE_LEFT && side != SSN_SIDE_RIGHT) return SSN_ERR_DTYPE;
   if (count < 0) return SSN_ERR_SHAPE;
   if (count == 0) return SSN_OK;
-  if (W_ptrs == nullptr || rows == nullptr || ldw == nullptr) return SSN_ERR_NULL;
+  if (W_ptrs == nullptr || extent == nullptr || ldw == nullptr) return SSN_ERR_NULL;
   for (int32_t b = 0; b < count; ++b) {
     if (W_ptrs[b] == nullptr) return SSN_ERR_NULL;
-    if (rows[b] < 1 || ldw[b] < codec->d) return SSN_ERR_SHAPE;
+    if (extent[b] < 1 || ldw[b] < (side == SSN_SIDE_RIGHT ? (int64_t)codec->d : extent[b])) return SSN_ERR_SHAPE;
   }
-  return reproject_right_list(codec, W_ptrs, rows, ldw, count, static_cast<cudaStream_t>(stream));
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (side == SSN_SIDE_RIGHT) return reproject_right_list(codec, W_ptrs, extent, ldw, count, s);
+  return reproject_left_list(codec, W_ptrs, extent, ldw, count, workspace, workspace_bytes, s);
 }
 
 ssn_status_t ssn_weight_reproject(const ssn_codec_t *codec, void *const *W_ptrs, int32_t batch,
@@ -365,31 +448,8 @@ ssn_status_t ssn_weight_reproject(const ssn_codec_t *codec, void *const *W_ptrs,
     return reproject_right_list(codec, W_ptrs, nrows.data(), lds.data(), batch, s);
   }
 
-  const int64_t col_blocks = (cols + kLeftCols - 1) / kLeftCols;
-  if (col_blocks > 0x7fffffffLL) return SSN_ERR_SHAPE;
-  for (int32_t b = 0; b < batch; ++b) {
-    LeftArgs a{};
-    a.W = W_ptrs[b];
-    a.U = codec->U;
-    a.T = static_cast<float *>(workspace);
-    a.ldw = ldw;
-    a.ldu = codec->ldu;
-    a.m = cols;
-    a.d = codec->d;
-    a.k = codec->k;
-    dim3 g1((unsigned)col_blocks, (unsigned)((codec->k + kGenericKChunk - 1) / kGenericKChunk));
-    dim3 g2((unsigned)col_blocks, (unsigned)((codec->d + 31) / 32));
-    if (codec->dtype == SSN_F32) {
-      left_reduce_kernel<float><<<g1, kLeftCols, 0, s>>>(a);
-      left_expand_kernel<float><<<g2, kLeftCols, 0, s>>>(a);
-    } else {
-      left_reduce_kernel<__nv_bfloat16><<<g1, kLeftCols, 0, s>>>(a);
-      left_expand_kernel<__nv_bfloat16><<<g2, kLeftCols, 0, s>>>(a);
-    }
-    st = launch_status(2);
-    if (st != SSN_OK) return st;
-  }
-  return SSN_OK;
+  std::vector<int64_t> ncols((size_t)batch, cols), lds((size_t)batch, ldw);
+  return reproject_left_list(codec, W_ptrs, ncols.data(), lds.data(), batch, workspace, workspace_bytes, s);
 }
 
 const char *ssn_status_string(ssn_status_t status) {

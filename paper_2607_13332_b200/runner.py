@@ -130,12 +130,25 @@ class Codec:
             return None
         return torch.empty(nbytes, dtype=torch.uint8, device=self.U.device)
 
+    def weight_reproject_list(self, weights: Sequence[torch.Tensor], side: str = "right",
+                              workspace: Optional[torch.Tensor] = None) -> None:
+        """In place, for weights [rows_i x d] ("right") or [d x cols_i] ("left") of any free
+        extents.  A LEFT weight the fused kernel does not take needs k * cols * 4 bytes of workspace;
+        one is allocated here when none is given."""
+        if not weights:
+            return
+        axis = 0 if side == "right" else 1
+        if side == "left" and workspace is None:
+            workspace = torch.empty(self.k * max(w.shape[1] for w in weights) * 4, dtype=torch.uint8,
+                                    device=self.U.device)
+        binding.ssn_weight_reproject_list(self.c, [w.data_ptr() for w in weights],
+                                          [w.shape[axis] for w in weights], [_ld(w) for w in weights],
+                                          binding.SIDES[side],
+                                          workspace.data_ptr() if workspace is not None else 0,
+                                          workspace.numel() if workspace is not None else 0, _stream())
+
     def weight_reproject_rows(self, weights: Sequence[torch.Tensor]) -> None:
-        """In place, RIGHT side, for weights [rows_i x d] of any row counts."""
-        if weights:
-            binding.ssn_weight_reproject_rows(self.c, [w.data_ptr() for w in weights],
-                                              [w.shape[0] for w in weights], [_ld(w) for w in weights],
-                                              _stream())
+        self.weight_reproject_list(weights, "right")
 
     def weight_reproject(self, weights: Sequence[torch.Tensor], side: str,
                          workspace: Optional[torch.Tensor] = None) -> None:

@@ -172,17 +172,68 @@ def test_reproject_rows_list_of_unequal_weights():
             assert_close(host64(w, dt2), oracle.weight_reproject(f64(w0, dt2), f64(U2, dt2), "right"), dt2, "general")
 
 
-def test_reproject_rows_argument_errors():
+def test_reproject_list_left_side_unequal_columns():
+    """LEFT side (W stored [d x m]): several weights of different widths in one call, in place,
+    at sizes that take the fused kernel and at ones that take the general one."""
+    dt, d, k = synth.BF16, 512, 40
+    U0 = synth.to_storage(synth.subspace_basis(d, k, seed=5), dt)
+    codec = Codec(dt, to_device(U0, dt))
+    U = f64(U0, dt)
+    cols = [512, 136, 1000, 8, 2048, 264, 128, 640, 72]
+    W0s = [synth.to_storage(np.random.default_rng(c).standard_normal((d, c)) * 0.05, dt) for c in cols]
+    views = [padded(d, c, c + 8 * (i % 3), dt, fill=to_device(w, dt)) for i, (c, w) in enumerate(zip(cols, W0s))]
+    codec.weight_reproject_list([v for v, _ in views], "left")
+    for (v, buf), w0 in zip(views, W0s):
+        assert_close(host64(v, dt), oracle.weight_reproject(f64(w0, dt), U, "left"), dt, f"cols {v.shape[1]}")
+        assert guards_intact(v, buf, dt)
+    # odd widths and leading dimensions, fp32: the general kernels through the workspace
+    for dt2, k2, widths in ((synth.BF16, 40, (333, 77)), (synth.F32, 24, (600, 50)), (synth.BF16, 72, (256,))):
+        U2 = synth.to_storage(synth.subspace_basis(d, k2, seed=6), dt2)
+        c2 = Codec(dt2, to_device(U2, dt2))
+        Ws0 = [synth.to_storage(np.random.default_rng(c).standard_normal((d, c)) * 0.05, dt2) for c in widths]
+        Ws = [to_device(w, dt2) for w in Ws0]
+        c2.weight_reproject_list(Ws, "left")
+        for w, w0 in zip(Ws, Ws0):
+            assert_close(host64(w, dt2), oracle.weight_reproject(f64(w0, dt2), f64(U2, dt2), "left"), dt2, "general")
+    # a weight that needs the workspace, without one
+    odd = to_device(Ws0[0], dt2)
+    with pytest.raises(binding.SsnError):
+        binding.ssn_weight_reproject_list(c2.c, [odd.data_ptr()], [odd.shape[1]], [odd.shape[1]],
+                                          binding.SIDES["left"])
+
+
+@pytest.mark.parametrize("k", [16, 40, 64])
+def test_left_reprojection_of_the_8b_shapes(k):
+    """The block's projections in the storage where the subspace is on the rows: out-proj
+    [4096 x 4096] and down-proj [4096 x 14336], one call."""
+    dt, d = synth.BF16, 4096
+    U0 = synth.to_storage(synth.subspace_basis(d, k, seed=50 + k), dt)
+    codec = Codec(dt, to_device(U0, dt))
+    W0s = [synth.projection_weight(d, m, seed=9, dtype=dt, layer=i) for i, m in enumerate((4096, 14336))]
+    Ws = [to_device(w, dt) for w in W0s]
+    codec.weight_reproject_list(Ws, "left")
+    for w, w0 in zip(Ws, W0s):
+        assert_close(host64(w, dt), oracle.weight_reproject(f64(w0, dt), f64(U0, dt), "left"), dt, f"left k={k}")
+
+
+def test_reproject_list_argument_errors():
     import ctypes
     dt, d, k = synth.BF16, 256, 8
     codec = Codec(dt, to_device(synth.to_storage(synth.subspace_basis(d, k, seed=3), dt), dt))
     W = torch.zeros((16, d), dtype=torch.bfloat16, device="cuda")
-    fn = binding.raw("ssn_weight_reproject_rows")
+    fn = binding.raw("ssn_weight_reproject_list")
     ptrs, one = (ctypes.c_void_p * 1)(W.data_ptr()), ctypes.c_int64
-    assert fn(codec.c, ptrs, (one * 1)(16), (one * 1)(d), 1, None) == binding.SSN_OK
-    assert fn(codec.c, ptrs, (one * 1)(0), (one * 1)(d), 1, None) == binding.SSN_ERR_SHAPE
-    assert fn(codec.c, ptrs, (one * 1)(16), (one * 1)(d - 1), 1, None) == binding.SSN_ERR_SHAPE
-    assert fn(codec.c, None, (one * 1)(16), (one * 1)(d), 1, None) == binding.SSN_ERR_NULL
-    assert fn(codec.c, (ctypes.c_void_p * 1)(None), (one * 1)(16), (one * 1)(d), 1, None) == binding.SSN_ERR_NULL
-    assert fn(codec.c, ptrs, (one * 1)(16), (one * 1)(d), 0, None) == binding.SSN_OK
-    assert fn(codec.c, ptrs, (one * 1)(16), (one * 1)(d), -1, None) == binding.SSN_ERR_SHAPE
+    R = binding.SIDES["right"]
+    assert fn(codec.c, ptrs, (one * 1)(16), (one * 1)(d), 1, R, None, 0, None) == binding.SSN_OK
+    assert fn(codec.c, ptrs, (one * 1)(0), (one * 1)(d), 1, R, None, 0, None) == binding.SSN_ERR_SHAPE
+    assert fn(codec.c, ptrs, (one * 1)(16), (one * 1)(d - 1), 1, R, None, 0, None) == binding.SSN_ERR_SHAPE
+    assert fn(codec.c, None, (one * 1)(16), (one * 1)(d), 1, R, None, 0, None) == binding.SSN_ERR_NULL
+    assert fn(codec.c, (ctypes.c_void_p * 1)(None), (one * 1)(16), (one * 1)(d), 1, R, None, 0, None) == binding.SSN_ERR_NULL
+    assert fn(codec.c, ptrs, (one * 1)(16), (one * 1)(d), 0, R, None, 0, None) == binding.SSN_OK
+    assert fn(codec.c, ptrs, (one * 1)(16), (one * 1)(d), -1, R, None, 0, None) == binding.SSN_ERR_SHAPE
+    assert fn(codec.c, ptrs, (one * 1)(16), (one * 1)(d), 1, 7, None, 0, None) == binding.SSN_ERR_DTYPE
+    L = binding.SIDES["left"]
+    Wl = torch.zeros((d, 24), dtype=torch.bfloat16, device="cuda")
+    pl = (ctypes.c_void_p * 1)(Wl.data_ptr())
+    assert fn(codec.c, pl, (one * 1)(24), (one * 1)(23), 1, L, None, 0, None) == binding.SSN_ERR_SHAPE
+    assert fn(codec.c, pl, (one * 1)(24), (one * 1)(24), 1, L, None, 0, None) == binding.SSN_ERR_WORKSPACE
