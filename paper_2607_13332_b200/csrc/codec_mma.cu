@@ -198,10 +198,27 @@ cudaError_t launch_umma_one(const MmaArgs &a, const UmmaMaps &maps, int sm_count
     if (e != cudaSuccess) return e;
     configured = true;
   }
-  int64_t grid = (a.n + kUmmaTile - 1) / kUmmaTile;
-  if (grid > sm_count) grid = sm_count;
-  kernel<<<(unsigned)grid, kUmmaThreads, smem, stream>>>(a, maps);
-  return cudaGetLastError();
+  // pairs of CTAs (clusters of two) that share their odd tile; see the kernel's schedule
+  const int64_t ntiles = (a.n + kUmmaTile - 1) / kUmmaTile;
+  int64_t pairs = (ntiles + 1) / 2;
+  if (pairs > sm_count / 2) pairs = sm_count / 2;
+  if (pairs < 1) {   // a single SM: plain launch
+    kernel<<<(unsigned)(ntiles < sm_count ? ntiles : sm_count), kUmmaThreads, smem, stream>>>(a, maps);
+    return cudaGetLastError();
+  }
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)(2 * pairs));
+  cfg.blockDim = dim3(kUmmaThreads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, a, maps);
 }
 
 template <int NTP>

@@ -60,6 +60,21 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
     if (++spins > kWaitSpins) return false;
   return true;
 }
+// The same with cluster-scope acquire: the phase was completed by arrivals from the peer CTA
+// that follow its writes into this CTA's shared memory.
+__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity) {
+  int spins = 0;
+  for (;;) {
+    uint32_t ok;
+    asm volatile(
+        "{\n.reg .pred p;\n"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n"
+        "selp.u32 %0, 1, 0, p;\n}\n"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    if (ok) return true;
+    if (++spins > kWaitSpins) return false;
+  }
+}
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, uint32_t bar,
                                             int c0, int c1) {
   asm volatile(
@@ -106,6 +121,11 @@ __device__ __forceinline__ uint64_t umma_desc(uint32_t addr, uint32_t lbo_bytes,
          ((uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32) | (1ull << 46) | ((uint64_t)layout_type << 61);
 }
 
+// Start-address field of a descriptor (14 bits, address / 16).  The mask matters: in a cluster
+// launch the shared-memory addresses of the CTAs of rank > 0 carry high bits, which would
+// otherwise spill into the neighbouring fields when the address is added to a prebuilt descriptor.
+__device__ __forceinline__ uint64_t umma_desc_addr(uint32_t addr) { return (uint64_t)((addr >> 4) & 0x3FFFu); }
+
 // Instruction descriptor: fp32 accumulate, bf16 A (K-major, optionally negated) and bf16 B
 // (MN-major), N and M encoded as N/8 and M/16.
 __host__ __device__ constexpr uint32_t umma_idesc(int n, bool negate_a) {
@@ -134,7 +154,7 @@ struct UmmaProjectConfig {
   static constexpr int kBufs = 2 * kIssuers * kAccCols <= 512 ? 2 : 1;   // accumulator sets (tiles in flight)
   static constexpr int kTmemCols = (kBufs * kIssuers * kAccCols) <= 128 ? 128 : ((kBufs * kIssuers * kAccCols) <= 256 ? 256 : 512);
   static_assert(kBufs * kIssuers * kAccCols <= 512, "accumulators do not fit in tensor memory");
-  static constexpr int kBarBytes = (2 * kStagesN + 4) * 8 + 16;
+  static constexpr int kBarBytes = (2 * kStagesN + 6) * 8 + 16;
   static constexpr int kSmemBytes = 1024 + kStagesN * kStageBytes + kBarBytes;
 };
 
@@ -164,11 +184,39 @@ codec_umma_project_kernel(const MmaArgs a, const __grid_constant__ UmmaMaps maps
   auto empty_bar = [&](int s) { return bars + (S + s) * 8; };
   auto acc_full_bar = [&](int b) { return bars + (2 * S + b) * 8; };
   auto acc_empty_bar = [&](int b) { return bars + (2 * S + 2 + b) * 8; };
-  const uint32_t tmem_slot = bars + (2 * S + 4) * 8;
+  const uint32_t partial_ready_bar = bars + (2 * S + 4) * 8;   // pair schedule: the peer's partial sums have arrived
+  const uint32_t ring_free_bar = bars + (2 * S + 5) * 8;       // pair schedule: the peer's stage ring may be overwritten
+  const uint32_t tmem_slot = bars + (2 * S + 6) * 8;
   volatile uint32_t *tmem_slot_ptr =
       reinterpret_cast<volatile uint32_t *>(smem_raw + (tmem_slot - smem_u32(smem_raw)));
 
+  // Tile schedule.  The CTAs run as pairs (clusters of two).  Pair c takes the tiles c, c + pairs,
+  // c + 2 pairs, ...; its two CTAs take them alternately, and when their number is odd the last
+  // tile is SPLIT: rank 0 contracts the first half of d, rank 1 the second half, rank 1 sends its
+  // fp32 partial sums into rank 0's (by then idle) stage ring through distributed shared memory,
+  // and rank 0 adds them and stores.  512 tiles on 74 pairs are 3 or 3.5 tiles per CTA instead of
+  // 3 or 4.  A launch without clusters is the same schedule with pairs of one CTA and no split.
+  uint32_t cluster_size, cta_rank;
+  asm volatile("mov.u32 %0, %%cluster_nctaid.x;\n" : "=r"(cluster_size));
+  asm volatile("mov.u32 %0, %%cluster_ctarank;\n" : "=r"(cta_rank));
+  const int64_t pairs = gridDim.x / cluster_size, pair = blockIdx.x / cluster_size;
+  const int64_t pair_tiles = pair < ntiles ? (ntiles - pair + pairs - 1) / pairs : 0;
+  const bool has_split = cluster_size == 2 && (pair_tiles & 1) && nstage >= 2;
+  const int my_tiles = (int)(cluster_size == 2
+                                 ? pair_tiles / 2 + (((pair_tiles & 1) && (has_split || cta_rank == 0)) ? 1 : 0)
+                                 : pair_tiles);
+  // i-th tile of this CTA: index, stage range, whether it is the split one
+  auto schedule = [&](int i, int64_t &tile, int &st_lo, int &st_hi, bool &split) {
+    split = has_split && i == my_tiles - 1;
+    const int64_t j = cluster_size == 2 ? (split ? pair_tiles - 1 : 2 * (int64_t)i + cta_rank) : i;
+    tile = pair + j * pairs;
+    st_lo = split && cta_rank == 1 ? nstage / 2 : 0;
+    st_hi = split && cta_rank == 0 ? nstage / 2 : nstage;
+  };
+
   if (threadIdx.x == 0) {
+    mbar_init(partial_ready_bar, 128);
+    mbar_init(ring_free_bar, 4);
     for (int s = 0; s < S; ++s) {
       mbar_init(full_bar(s), HAS_E ? 5 : 1);
       mbar_init(empty_bar(s), Cfg::kIssuers);
@@ -186,6 +234,8 @@ codec_umma_project_kernel(const MmaArgs a, const __grid_constant__ UmmaMaps maps
   }
   asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
   __syncthreads();
+  // the peer's barriers must exist before anything arrives on them
+  asm volatile("barrier.cluster.arrive.release.aligned;\nbarrier.cluster.wait.acquire.aligned;\n" ::: "memory");
   asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
   const uint32_t tmem_base = *tmem_slot_ptr;
   bool dead = false;
@@ -198,10 +248,14 @@ codec_umma_project_kernel(const MmaArgs a, const __grid_constant__ UmmaMaps maps
     // ------------------------------------------------------------------------- producer
     int slot = 0;
     uint32_t parity = 1;   // a fresh "empty" barrier passes a wait on parity 1
-    for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+    for (int it = 0; it < my_tiles; ++it) {
+      int64_t tile;
+      int st_lo, st_hi;
+      bool split;
+      schedule(it, tile, st_lo, st_hi, split);
       const int64_t tok0 = tile * kUmmaTile;
       const int pos0 = HAS_P ? (int)(tok0 % a.shift.seq_len) : 0;
-      for (int st = 0; st < nstage; ++st) {
+      for (int st = st_lo; st < st_hi; ++st) {
         if (!dead && !mbar_wait(empty_bar(slot), parity)) timed_out();
         const uint32_t base = smem0 + (uint32_t)slot * Cfg::kStageBytes;
         const uint32_t bar = full_bar(slot);
@@ -236,25 +290,29 @@ codec_umma_project_kernel(const MmaArgs a, const __grid_constant__ UmmaMaps maps
       int slot = 0;
       uint32_t parity = 0;
       int64_t tcount = 0;
-      for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x, ++tcount) {
+      for (int it = 0; it < my_tiles; ++it, ++tcount) {
+        int64_t tile;
+        int st_lo, st_hi;
+        bool split;
+        schedule(it, tile, st_lo, st_hi, split);
         const int buf = (int)(tcount % Cfg::kBufs);
         const uint32_t acc_parity = (uint32_t)((tcount / Cfg::kBufs) & 1);
         if (!dead && !mbar_wait(acc_empty_bar(buf), acc_parity ^ 1u)) timed_out();
         asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
         const uint32_t d_tmem = tmem_base + (uint32_t)(buf * Cfg::kIssuers + which) * Cfg::kAccCols;
-        for (int st = 0; st < nstage; ++st) {
+        for (int st = st_lo; st < st_hi; ++st) {
           if (!dead && !mbar_wait(full_bar(slot), parity)) timed_out();
           asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
           const uint32_t base = smem0 + (uint32_t)slot * Cfg::kStageBytes;
           // the start-address field (address / 16) is added to descriptors built once: a K step
           // is 32 bytes of an A row and 16 rows = 2048 bytes of the U slice
-          const uint64_t adesc = adesc0 + ((base + (uint32_t)which * Cfg::kATileBytes) >> 4);
-          const uint64_t bdesc = bdesc0 + ((base + Cfg::kATiles * Cfg::kATileBytes) >> 4);
+          const uint64_t adesc = adesc0 + umma_desc_addr(base + (uint32_t)which * Cfg::kATileBytes);
+          const uint64_t bdesc = bdesc0 + umma_desc_addr(base + Cfg::kATiles * Cfg::kATileBytes);
 #pragma unroll
           for (int j = 0; j < kUmmaCols / 16; ++j)
-            umma_bf16(d_tmem, adesc + j * 2, bdesc + j * 128, idesc, (st > 0 || j > 0) ? 1u : 0u);
+            umma_bf16(d_tmem, adesc + j * 2, bdesc + j * 128, idesc, (st > st_lo || j > 0) ? 1u : 0u);
           umma_commit(empty_bar(slot));
-          if (st == nstage - 1) umma_commit(acc_full_bar(buf));
+          if (st == st_hi - 1) umma_commit(acc_full_bar(buf));
           if (++slot == S) {
             slot = 0;
             parity ^= 1u;
@@ -276,7 +334,11 @@ codec_umma_project_kernel(const MmaArgs a, const __grid_constant__ UmmaMaps maps
         if (++pub_slot == S) pub_slot = 0;
         --pending;
       };
-      for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+      for (int it = 0; it < my_tiles; ++it) {
+        int64_t tile;
+        int st_lo, st_hi;
+        bool split;
+        schedule(it, tile, st_lo, st_hi, split);
         const int64_t tok0 = tile * kUmmaTile;
         const unsigned char *src[8];
         uint32_t dst[8];
@@ -290,7 +352,7 @@ codec_umma_project_kernel(const MmaArgs a, const __grid_constant__ UmmaMaps maps
                             : g_zero_row) + piece * 16;
           dst[i] = kETile * Cfg::kATileBytes + r * 128 + ((piece ^ (r & 7)) << 4);
         }
-        for (int st = 0; st < nstage; ++st) {
+        for (int st = st_lo; st < st_hi; ++st) {
           if (!dead && !mbar_wait(empty_bar(slot), parity)) timed_out();
           const uint32_t base = smem0 + (uint32_t)slot * Cfg::kStageBytes;
 #pragma unroll
@@ -314,7 +376,11 @@ codec_umma_project_kernel(const MmaArgs a, const __grid_constant__ UmmaMaps maps
     const int quarter = warp & 3;   // the TMEM lanes this warp may read: 32*quarter .. +31
     int64_t tcount = 0;
     const bool vec = ((a.ldzout & 7) == 0) && ((reinterpret_cast<uintptr_t>(a.zout) & 15) == 0);
-    for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x, ++tcount) {
+    for (int it = 0; it < my_tiles; ++it, ++tcount) {
+      int64_t tile;
+      int st_lo, st_hi;
+      bool split;
+      schedule(it, tile, st_lo, st_hi, split);
       const int buf = (int)(tcount % Cfg::kBufs);
       const uint32_t acc_parity = (uint32_t)((tcount / Cfg::kBufs) & 1);
       if (!dead && !mbar_wait(acc_full_bar(buf), acc_parity)) timed_out();
@@ -339,6 +405,45 @@ codec_umma_project_kernel(const MmaArgs a, const __grid_constant__ UmmaMaps maps
       asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
       __syncwarp();
       if (lane == 0) mbar_arrive(acc_empty_bar(buf));
+
+      if (split) {
+        // the split tile is the last one of both CTAs: every stage of rank 0's ring has been
+        // consumed once its accumulator is complete, so the ring can carry the partial sums
+        const uint32_t row_off = (uint32_t)(quarter * 32 + lane) * (Cfg::kN * 4);
+        if (cta_rank == 0) {
+          if (lane == 0) {
+            uint32_t remote;
+            asm volatile("mapa.shared::cluster.u32 %0, %1, %2;\n" : "=r"(remote) : "r"(ring_free_bar), "r"(1));
+            asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];\n" ::"r"(remote) : "memory");
+          }
+          if (!dead && !mbar_wait_cluster(partial_ready_bar, 0)) timed_out();
+#pragma unroll
+          for (int q = 0; q < Cfg::kN / 16; ++q)
+#pragma unroll
+            for (int i = 0; i < 16; i += 4) {
+              float4 w;
+              asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];\n"
+                           : "=f"(w.x), "=f"(w.y), "=f"(w.z), "=f"(w.w) : "r"(smem0 + row_off + (q * 16 + i) * 4));
+              v[q][i] = __float_as_uint(__uint_as_float(v[q][i]) + w.x);
+              v[q][i + 1] = __float_as_uint(__uint_as_float(v[q][i + 1]) + w.y);
+              v[q][i + 2] = __float_as_uint(__uint_as_float(v[q][i + 2]) + w.z);
+              v[q][i + 3] = __float_as_uint(__uint_as_float(v[q][i + 3]) + w.w);
+            }
+        } else {
+          if (!dead && !mbar_wait_cluster(ring_free_bar, 0)) timed_out();
+          uint32_t remote_ring, remote_bar;
+          asm volatile("mapa.shared::cluster.u32 %0, %1, %2;\n" : "=r"(remote_ring) : "r"(smem0 + row_off), "r"(0));
+          asm volatile("mapa.shared::cluster.u32 %0, %1, %2;\n" : "=r"(remote_bar) : "r"(partial_ready_bar), "r"(0));
+#pragma unroll
+          for (int q = 0; q < Cfg::kN / 16; ++q)
+#pragma unroll
+            for (int i = 0; i < 16; i += 4)
+              asm volatile("st.shared::cluster.v4.b32 [%0], {%1,%2,%3,%4};\n" ::"r"(remote_ring + (q * 16 + i) * 4),
+                           "r"(v[q][i]), "r"(v[q][i + 1]), "r"(v[q][i + 2]), "r"(v[q][i + 3]) : "memory");
+          asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];\n" ::"r"(remote_bar) : "memory");
+          continue;   // rank 0 stores this tile
+        }
+      }
 
       const int64_t t = tile * kUmmaTile + quarter * 32 + lane;
       if (t < a.n) {
@@ -390,6 +495,8 @@ codec_umma_project_kernel(const MmaArgs a, const __grid_constant__ UmmaMaps maps
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem_base),
                  "r"(Cfg::kTmemCols) : "memory");
   }
+  // neither CTA of a pair may leave while the other can still touch its shared memory
+  asm volatile("barrier.cluster.arrive.release.aligned;\nbarrier.cluster.wait.acquire.aligned;\n" ::: "memory");
 }
 
 }  // namespace ssn

@@ -223,14 +223,14 @@ codec_umma_expand_kernel(const MmaArgs a, const ExpandGeometry geo, const __grid
       constexpr uint32_t idesc_kmn = umma_idesc(kChunkCols, false);       // Sel (K-major) x P rows (MN-major)
       const uint64_t kdesc = umma_desc(0, 16, 1024, 2);
       const uint64_t pdesc = umma_desc(0, kGridPos * 128, 1024, 2);       // 64-column groups 2048 bytes apart
-      const uint64_t seld = kdesc + (sel >> 4);
+      const uint64_t seld = kdesc + umma_desc_addr(sel);
       int slot = 0;
       uint32_t parity = 0;
       int64_t tcount = 0, ccount = 0;
       for (int64_t tile = tile_lo; tile <= tile_hi; ++tile, ++tcount) {
         const int zb = (int)(tcount & 1);
         if (!dead && !mbar_wait(z_full_bar(zb), (uint32_t)((tcount >> 1) & 1))) timed_out();
-        const uint64_t zd = kdesc + ((z_base + zb * Cfg::kTileBytes) >> 4);
+        const uint64_t zd = kdesc + umma_desc_addr(z_base + zb * Cfg::kTileBytes);
         int q0, q1;
         chunk_range(tile, q0, q1);
         for (int q = q0; q < q1; ++q, ++ccount) {
@@ -240,9 +240,9 @@ codec_umma_expand_kernel(const MmaArgs a, const ExpandGeometry geo, const __grid
           asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
           const uint32_t base = u_ring + (uint32_t)slot * Cfg::kUStageBytes;
           const uint32_t dacc = tmem_base + (uint32_t)db * kChunkCols;
-          const uint64_t bd = kdesc + (base >> 4);
+          const uint64_t bd = kdesc + umma_desc_addr(base);
           for (int j = 0; j < ksteps; ++j) umma_bf16(dacc, zd + j * 2, bd + j * 2, idesc_kk, j > 0 ? 1u : 0u);
-          if (HAS_P) umma_bf16(dacc, seld, pdesc + ((base + Cfg::kU2Bytes) >> 4), idesc_kmn, 1u);
+          if (HAS_P) umma_bf16(dacc, seld, pdesc + umma_desc_addr(base + Cfg::kU2Bytes), idesc_kmn, 1u);
           umma_commit(u_empty_bar(slot));
           umma_commit(d_full_bar(db));
           if (q == q1 - 1) umma_commit(z_empty_bar(zb));

@@ -227,7 +227,7 @@ codec_umma_roundtrip_kernel(const MmaArgs a, const __grid_constant__ UmmaRoundTr
           if (!dead && !mbar_wait(full_bar(slot), parity)) timed_out();
           asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
           const uint32_t base = ring + (uint32_t)slot * Cfg::kStageBytes;
-          const uint64_t ad = (LEFT ? wdesc : kdesc) + (base >> 4), bd = udesc + ((base + Cfg::kTileBytes) >> 4);
+          const uint64_t ad = (LEFT ? wdesc : kdesc) + umma_desc_addr(base), bd = udesc + umma_desc_addr(base + Cfg::kTileBytes);
 #pragma unroll
           for (int j = 0; j < kUmmaCols / 16; ++j)   // a K step: 32 bytes of a K-major row, 16 rows of an MN-major tile
             umma_bf16(acc1, ad + j * (LEFT ? 128 : 2), bd + j * 128, idesc1, (st > 0 || j > 0) ? 1u : 0u);
@@ -246,8 +246,8 @@ codec_umma_roundtrip_kernel(const MmaArgs a, const __grid_constant__ UmmaRoundTr
           if (!dead && !mbar_wait(u2_full_bar(uslot), uparity)) timed_out();
           asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
           const uint32_t dacc = tmem_base + Cfg::kDCol + (uint32_t)db * kChunkCols;
-          const uint64_t bd = kdesc + ((u2_ring + (uint32_t)uslot * Cfg::kU2Bytes) >> 4);
-          const uint64_t hd = kdesc + (c_hi >> 4), ld = kdesc + (c_lo >> 4);
+          const uint64_t bd = kdesc + umma_desc_addr(u2_ring + (uint32_t)uslot * Cfg::kU2Bytes);
+          const uint64_t hd = kdesc + umma_desc_addr(c_hi), ld = kdesc + umma_desc_addr(c_lo);
 #pragma unroll
           for (int j = 0; j < Cfg::kKSteps; ++j) {
             if (LEFT) {   // rows of U times the coordinates of the column block

@@ -26,6 +26,9 @@ SHAPES = [
     (3, 333, 256, 24, 77),       # sequence length not a multiple of 16
     (16, 64, 192, 40, 60),       # d not a multiple of 128
     (16, 64, 256, 72, 60),       # k > 64
+    (12, 256, 2048, 128, 999),   # k = 128: two column groups of U; 24 tiles on 12 CTA pairs
+    (17, 128, 1024, 96, 500),    # 17 tiles: the last pair splits its tile over d
+    (1, 640, 512, 40, 200),      # 5 tiles on 3 pairs, one of them split
 ]
 
 
