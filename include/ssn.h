@@ -175,7 +175,7 @@ ssn_status_t ssn_weight_reproject(const ssn_codec_t *codec, void *const *W_ptrs,
  *   W_ptrs, extent, ldw   HOST arrays of `count` device pointers, extents (>= 1) and leading
  *                         dimensions (>= d for RIGHT, >= extent[i] for LEFT); distinct buffers.
  *   workspace   only read for SSN_SIDE_LEFT weights that the fused tensor-core kernel does not
- *               take (fp32, k > 64, d not a multiple of 128, leading dimension not a multiple of
+ *               take (fp32, k > 128, d not a multiple of 128, leading dimension not a multiple of
  *               8 elements, unaligned base): k * max(extent) * 4 bytes, 16-byte aligned; such a
  *               weight without enough workspace gives SSN_ERR_WORKSPACE (weights before it in the
  *               list have been re-projected then).  May be NULL otherwise.

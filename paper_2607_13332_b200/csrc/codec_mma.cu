@@ -284,14 +284,14 @@ cudaError_t launch_roundtrip_ntp(const MmaArgs &a, const UmmaRoundTripMaps &maps
 
 // Project-then-expand on tcgen05 for `count` matrices [rows[i] x d] at once (src[i] -> dst[i], which
 // may be the same buffer).  Returns cudaErrorNotSupported when the call should take the mma.sync
-// kernels instead: k > 64, d not a multiple of 128, few rows in all, too many matrices, no tensor map
+// kernels instead: k > 128, d not a multiple of 128, few rows in all, too many matrices, no tensor map
 // (unaligned base or leading dimension).  zout (coordinates, bf16) only with one matrix.
 cudaError_t launch_codec_umma_roundtrip_list(const MmaArgs &a, const __nv_bfloat16 *const *src,
                                              __nv_bfloat16 *const *dst, const int64_t *rows,
                                              const int64_t *lds, const int64_t *lddst, int count,
                                              int sm_count, cudaStream_t stream, bool left) {
   if (count < 1 || count > kRoundTripMaxMatrices) return cudaErrorNotSupported;
-  if (a.d % kChunkCols != 0 || a.k > 64) return cudaErrorNotSupported;
+  if (a.d % kChunkCols != 0 || a.k > 128) return cudaErrorNotSupported;
   UmmaRoundTripMaps maps;
   int64_t tiles = 0, total = 0;
   for (int i = 0; i < count; ++i) {
@@ -319,7 +319,7 @@ cudaError_t launch_codec_umma_roundtrip_list(const MmaArgs &a, const __nv_bfloat
   maps.tile_start[count] = (int32_t)tiles;
   maps.count = count;
   if (!make_sw128_map(&maps.u, a.U, a.d, a.k, a.ldu, kUmmaCols)) return cudaErrorNotSupported;
-  if (!make_sw128_map(&maps.u_wide, a.U, a.d, 64, a.ldu, kUmmaCols)) return cudaErrorNotSupported;
+  if (!make_sw128_map(&maps.u_wide, a.U, a.d, a.k <= 64 ? 64 : 128, a.ldu, kUmmaCols)) return cudaErrorNotSupported;
   MmaArgs b = a;
   if (count > 1 || left) b.zout = nullptr;
   const int ntp = 2 * ((a.k + 15) / 16);
@@ -327,12 +327,16 @@ cudaError_t launch_codec_umma_roundtrip_list(const MmaArgs &a, const __nv_bfloat
     if (ntp <= 2) return launch_roundtrip_ntp<2, true>(b, maps, sm_count, stream);
     if (ntp <= 4) return launch_roundtrip_ntp<4, true>(b, maps, sm_count, stream);
     if (ntp <= 6) return launch_roundtrip_ntp<6, true>(b, maps, sm_count, stream);
-    return launch_roundtrip_ntp<8, true>(b, maps, sm_count, stream);
+    if (ntp <= 8) return launch_roundtrip_ntp<8, true>(b, maps, sm_count, stream);
+    if (ntp <= 12) return launch_roundtrip_ntp<12, true>(b, maps, sm_count, stream);
+    return launch_roundtrip_ntp<16, true>(b, maps, sm_count, stream);
   }
   if (ntp <= 2) return launch_roundtrip_ntp<2, false>(b, maps, sm_count, stream);
   if (ntp <= 4) return launch_roundtrip_ntp<4, false>(b, maps, sm_count, stream);
   if (ntp <= 6) return launch_roundtrip_ntp<6, false>(b, maps, sm_count, stream);
-  return launch_roundtrip_ntp<8, false>(b, maps, sm_count, stream);
+  if (ntp <= 8) return launch_roundtrip_ntp<8, false>(b, maps, sm_count, stream);
+  if (ntp <= 12) return launch_roundtrip_ntp<12, false>(b, maps, sm_count, stream);
+  return launch_roundtrip_ntp<16, false>(b, maps, sm_count, stream);
 }
 
 cudaError_t launch_codec_umma_roundtrip(const MmaArgs &a, int sm_count, cudaStream_t stream) {

@@ -1,4 +1,4 @@
-// tcgen05 / TMA "project then expand" kernel of the SSN codec (bf16, sm_100a), k <= 64:
+// tcgen05 / TMA "project then expand" kernel of the SSN codec (bf16, sm_100a), k <= 128:
 //     C = S U   (fp32, in tensor memory),   D = C U^T        S, D: [n x d]
 // used for the weight re-projection W <- (W U) U^T of the original SSN (Sec. 4.1; S and D are
 // then the same buffer) and for the projected gradient G U U^T.  A tile of 128 rows is read
@@ -57,16 +57,19 @@ __host__ __device__ constexpr uint32_t umma_idesc_kk(int n) {
 
 template <int NTP>
 struct UmmaRoundTripConfig {
-  static_assert(NTP % 2 == 0 && NTP >= 2 && NTP <= 8, "N = 8*NTP must be a multiple of 16 up to 64");
+  static_assert(NTP % 2 == 0 && NTP >= 2 && NTP <= 16, "N = 8*NTP must be a multiple of 16 up to 128");
   static constexpr int kN = NTP * 8;
+  static constexpr int kKG = kN <= 64 ? 1 : 2;                  // 64-coordinate groups (128-byte operand rows)
   static constexpr int kKSteps = kN / 16;                       // K steps of pass 2
   static constexpr int kTileBytes = kUmmaTile * 128;            // [128 rows x 128 B]
-  static constexpr int kUBytes = kUmmaCols * 128;               // pass 1: 64 rows of U
+  static constexpr int kUGroupBytes = kUmmaCols * 128;          // pass 1: 64 rows of U, one 64-column group
+  static constexpr int kUBytes = kKG * kUGroupBytes;
   static constexpr int kStageBytes = kTileBytes + kUBytes;
-  static constexpr int kU2Bytes = kChunkCols * 128;             // pass 2: 128 rows of U, K-major
+  static constexpr int kCBytes = kKG * kTileBytes;              // the coordinates as an operand: [128 x k]
+  static constexpr int kU2Bytes = kKG * kChunkCols * 128;       // pass 2: 128 rows of U, K-major
   static constexpr int kU2Stages = 2;
   static constexpr int kStagingBytes = 4 * 2 * 4096;            // per epilogue warp two [32 x 128 B] slabs
-  static constexpr int kFixedBytes = 2 * kTileBytes + kU2Stages * kU2Bytes + kStagingBytes;
+  static constexpr int kFixedBytes = 2 * kCBytes + kU2Stages * kU2Bytes + kStagingBytes;
   static constexpr int kMaxSmem = 227 * 1024;
   static constexpr int kFit = (kMaxSmem - 1024 - 512 - kFixedBytes) / kStageBytes;
   static constexpr int kStagesN = kFit < 8 ? kFit : 8;
@@ -110,8 +113,8 @@ codec_umma_roundtrip_kernel(const MmaArgs a, const __grid_constant__ UmmaRoundTr
   };
 
   const uint32_t smem0 = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  const uint32_t c_hi = smem0, c_lo = smem0 + Cfg::kTileBytes;
-  const uint32_t u2_ring = c_lo + Cfg::kTileBytes;
+  const uint32_t c_hi = smem0, c_lo = smem0 + Cfg::kCBytes;
+  const uint32_t u2_ring = c_lo + Cfg::kCBytes;
   const uint32_t staging = u2_ring + S2 * Cfg::kU2Bytes;
   const uint32_t ring = staging + Cfg::kStagingBytes;
   const uint32_t bars = ring + S * Cfg::kStageBytes;
@@ -177,8 +180,10 @@ codec_umma_roundtrip_kernel(const MmaArgs a, const __grid_constant__ UmmaRoundTr
           } else {
             tma_load_2d(base, &maps.s[w], full_bar(slot), st * kUmmaCols, row0);
           }
-          tma_load_2d(base + Cfg::kTileBytes, st == nstage - 1 ? &maps.u : &maps.u_wide, full_bar(slot), 0,
-                      st * kUmmaCols);
+#pragma unroll
+          for (int ug = 0; ug < Cfg::kKG; ++ug)
+            tma_load_2d(base + Cfg::kTileBytes + ug * Cfg::kUGroupBytes, st == nstage - 1 ? &maps.u : &maps.u_wide,
+                        full_bar(slot), ug * 64, st * kUmmaCols);
         }
         __syncwarp();
         if (++slot == S) {
@@ -197,9 +202,12 @@ codec_umma_roundtrip_kernel(const MmaArgs a, const __grid_constant__ UmmaRoundTr
         const uint32_t base = u2_ring + (uint32_t)slot * Cfg::kU2Bytes;
         if (lane == 0) {
           mbar_expect_tx(u2_full_bar(slot), Cfg::kU2Bytes);
-          tma_load_2d(base, &maps.u_wide, u2_full_bar(slot), 0, q * kChunkCols);
-          tma_load_2d(base + Cfg::kUBytes, q == nchunks - 1 ? &maps.u : &maps.u_wide, u2_full_bar(slot), 0,
-                      q * kChunkCols + kUmmaCols);
+#pragma unroll
+          for (int kg = 0; kg < Cfg::kKG; ++kg) {   // per 64-coordinate group: 128 rows of 128 bytes
+            tma_load_2d(base + kg * Cfg::kTileBytes, &maps.u_wide, u2_full_bar(slot), kg * 64, q * kChunkCols);
+            tma_load_2d(base + kg * Cfg::kTileBytes + Cfg::kUGroupBytes, q == nchunks - 1 ? &maps.u : &maps.u_wide,
+                        u2_full_bar(slot), kg * 64, q * kChunkCols + kUmmaCols);
+          }
         }
         __syncwarp();
         if (++slot == S2) {
@@ -216,7 +224,7 @@ codec_umma_roundtrip_kernel(const MmaArgs a, const __grid_constant__ UmmaRoundTr
       constexpr uint32_t idesc2 = umma_idesc_kk(kChunkCols);
       // descriptors without the start address, which is added per instruction (address / 16)
       const uint64_t kdesc = umma_desc(0, 16, 1024, 2);                 // K-major tile, rows of 128 B
-      const uint64_t udesc = umma_desc(0, Cfg::kUBytes, 1024, 2);       // U slice of pass 1 (MN-major)
+      const uint64_t udesc = umma_desc(0, Cfg::kUGroupBytes, 1024, 2);  // U slice of pass 1 (MN-major)
       const uint64_t wdesc = umma_desc(0, Cfg::kTileBytes / 2, 1024, 2);  // LEFT: W block, two 64-column groups
       int slot = 0, uslot = 0;
       uint32_t parity = 0, uparity = 0;
@@ -250,12 +258,14 @@ codec_umma_roundtrip_kernel(const MmaArgs a, const __grid_constant__ UmmaRoundTr
           const uint64_t hd = kdesc + umma_desc_addr(c_hi), ld = kdesc + umma_desc_addr(c_lo);
 #pragma unroll
           for (int j = 0; j < Cfg::kKSteps; ++j) {
+            // K step j: 32 bytes into the rows of 64-coordinate group j / 4
+            const uint32_t ko = (uint32_t)(j >> 2) * (Cfg::kTileBytes >> 4) + (uint32_t)(j & 3) * 2;
             if (LEFT) {   // rows of U times the coordinates of the column block
-              umma_bf16(dacc, bd + j * 2, hd + j * 2, idesc2, j > 0 ? 1u : 0u);
-              umma_bf16(dacc, bd + j * 2, ld + j * 2, idesc2, 1u);
+              umma_bf16(dacc, bd + ko, hd + ko, idesc2, j > 0 ? 1u : 0u);
+              umma_bf16(dacc, bd + ko, ld + ko, idesc2, 1u);
             } else {
-              umma_bf16(dacc, hd + j * 2, bd + j * 2, idesc2, j > 0 ? 1u : 0u);
-              umma_bf16(dacc, ld + j * 2, bd + j * 2, idesc2, 1u);
+              umma_bf16(dacc, hd + ko, bd + ko, idesc2, j > 0 ? 1u : 0u);
+              umma_bf16(dacc, ld + ko, bd + ko, idesc2, 1u);
             }
           }
           umma_commit(u2_empty_bar(uslot));
@@ -289,7 +299,7 @@ codec_umma_roundtrip_kernel(const MmaArgs a, const __grid_constant__ UmmaRoundTr
         asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
         const int64_t t = row0 + r;
 #pragma unroll
-        for (int c = 0; c < 8; ++c) {           // 16-byte pieces: 8 coordinates each
+        for (int c = 0; c < 8 * Cfg::kKG; ++c) {           // 16-byte pieces: 8 coordinates each
           uint32_t hi[4] = {0, 0, 0, 0}, lo[4] = {0, 0, 0, 0};
           if (c * 8 < Cfg::kN) {
 #pragma unroll
@@ -313,7 +323,8 @@ codec_umma_roundtrip_kernel(const MmaArgs a, const __grid_constant__ UmmaRoundTr
               }
             }
           }
-          const uint32_t off = (uint32_t)r * 128 + (uint32_t)((c ^ (r & 7)) << 4);
+          const uint32_t off = (uint32_t)(c >> 3) * Cfg::kTileBytes + (uint32_t)r * 128 +
+                               (uint32_t)(((c & 7) ^ (r & 7)) << 4);
           asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};\n" ::"r"(c_hi + off), "r"(hi[0]), "r"(hi[1]),
                        "r"(hi[2]), "r"(hi[3]) : "memory");
           asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};\n" ::"r"(c_lo + off), "r"(lo[0]), "r"(lo[1]),

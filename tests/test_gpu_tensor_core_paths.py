@@ -114,7 +114,8 @@ def test_prepare_tables_argument_errors():
 
 
 @pytest.mark.parametrize("rows,d,k", [(512, 256, 40), (1000, 512, 8), (2125, 1024, 64), (640, 384, 33),
-                                      (3000, 2048, 16), (4096, 4096, 40)])
+                                      (3000, 2048, 16), (4096, 4096, 40), (3000, 2048, 128), (1024, 512, 96),
+                                      (2000, 1024, 72)])
 def test_project_then_expand_in_place_with_guard_bands(rows, d, k):
     """Weight re-projection (in place) and the projected gradient (out of place, with the
     coordinates) at sizes that take the fused tcgen05 kernel; nothing outside the rows moves."""
@@ -190,7 +191,7 @@ def test_reproject_list_left_side_unequal_columns():
         assert_close(host64(v, dt), oracle.weight_reproject(f64(w0, dt), U, "left"), dt, f"cols {v.shape[1]}")
         assert guards_intact(v, buf, dt)
     # odd widths and leading dimensions, fp32: the general kernels through the workspace
-    for dt2, k2, widths in ((synth.BF16, 40, (333, 77)), (synth.F32, 24, (600, 50)), (synth.BF16, 72, (256,))):
+    for dt2, k2, widths in ((synth.BF16, 40, (333, 77)), (synth.F32, 24, (600, 50)), (synth.BF16, 136, (256,))):
         U2 = synth.to_storage(synth.subspace_basis(d, k2, seed=6), dt2)
         c2 = Codec(dt2, to_device(U2, dt2))
         Ws0 = [synth.to_storage(np.random.default_rng(c).standard_normal((d, c)) * 0.05, dt2) for c in widths]
@@ -205,7 +206,7 @@ def test_reproject_list_left_side_unequal_columns():
                                           binding.SIDES["left"])
 
 
-@pytest.mark.parametrize("k", [16, 40, 64])
+@pytest.mark.parametrize("k", [16, 40, 64, 128])
 def test_left_reprojection_of_the_8b_shapes(k):
     """The block's projections in the storage where the subspace is on the rows: out-proj
     [4096 x 4096] and down-proj [4096 x 14336], one call."""
