@@ -74,6 +74,14 @@ typedef enum { SSN_GRAD_COEFF = 1, SSN_GRAD_FULL = 2 } ssn_grad_mode_t;
  * The data both ends of a stage boundary share (Sec. 4.1: the basis U_k, and PE and T_fixed
  * "available to both sender and receiver").  Plain value struct; nothing is owned.
  */
+/*
+ * Performance note.  The tensor-core kernels need 16-byte aligned base addresses and leading
+ * dimensions that are multiples of 8 elements (bf16) for U, X / G / Xhat, E, P and the weights,
+ * and for Z where it is read (decompress).  A rank that is not a multiple of 8 (the paper's 8B
+ * run uses ~51) is fine as long as U and Z are STORED with such a leading dimension (ldu = 56,
+ * say; the padding columns are never read as data).  Anything else still gives the same results,
+ * through the general kernels, two orders of magnitude slower.
+ */
 typedef struct ssn_codec {
   int32_t d;            /* model width, >= 1                                              */
   int32_t k;            /* subspace rank, 1 <= k <= d                                     */

@@ -34,6 +34,17 @@ def to_host(t: torch.Tensor, dtype: str) -> np.ndarray:
     return t.detach().contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
 
 
+def padded_columns(t: torch.Tensor, multiple: int = 8) -> torch.Tensor:
+    """A copy of the 2-D tensor t whose leading dimension is rounded up to `multiple` elements,
+    returned as the [rows, cols] view of the padded buffer (zeros in the padding).  The
+    tensor-core kernels need such leading dimensions; see the note in include/ssn.h."""
+    rows, cols = t.shape
+    ld = -(-cols // multiple) * multiple
+    buf = torch.zeros((rows, ld), dtype=t.dtype, device=t.device)
+    buf[:, :cols] = t
+    return buf[:, :cols]
+
+
 def _stream() -> int:
     return torch.cuda.current_stream().cuda_stream
 

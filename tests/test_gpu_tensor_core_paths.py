@@ -241,3 +241,34 @@ def test_reproject_list_argument_errors():
     pl = (ctypes.c_void_p * 1)(Wl.data_ptr())
     assert fn(codec.c, pl, (one * 1)(24), (one * 1)(23), 1, L, None, 0, None) == binding.SSN_ERR_SHAPE
     assert fn(codec.c, pl, (one * 1)(24), (one * 1)(24), 1, L, None, 0, None) == binding.SSN_ERR_WORKSPACE
+
+
+def test_rank_that_is_not_a_multiple_of_8_with_padded_leading_dimensions():
+    """k = 51 (the rank of the paper's 8B run): with U and Z stored at a leading dimension of 56
+    every step takes the tensor-core kernels; results against the oracle, padding untouched."""
+    from paper_2607_13332_b200.runner import padded_columns
+    wl, t = _inputs(8, 256, 1024, 51, 300, seed=51)
+    dt, n = wl.dtype, wl.n_tokens
+    U = padded_columns(to_device(t["U"], dt))
+    assert U.stride(0) == 56
+    codec = Codec(dt, U, to_device(t["E"], dt), to_device(t["P"], dt))
+    ids = torch.from_numpy(t["ids"]).cuda()
+    Uf, Ef, Pf = f64(t["U"], dt), f64(t["E"], dt), f64(t["P"], dt)
+    pos = oracle.token_positions(n, wl.seq_len)
+    Zv, Zbuf = padded(n, wl.k, 56, dt)
+    codec.compress(to_device(t["X"], dt), ids, seq_len=wl.seq_len, out=Zv)
+    Zo, _ = oracle.compress(f64(t["X"], dt), Uf, Ef, t["ids"], Pf, pos)
+    assert_close(host64(Zv, dt), Zo, dt, "compress")
+    assert guards_intact(Zv, Zbuf, dt)
+    Z0v, _ = padded(n, wl.k, 56, dt, fill=to_device(t["Z0"], dt))
+    Xh = codec.decompress(Z0v, ids, seq_len=wl.seq_len)
+    Xo, _ = oracle.decompress(f64(t["Z0"], dt), Uf, Ef, t["ids"], Pf, pos)
+    assert_close(host64(Xh, dt), Xo, dt, "decompress")
+    dZ, Gp = codec.grad_project(to_device(t["G"], dt), full=True)
+    assert_close(host64(dZ, dt), oracle.grad_project_coeff(f64(t["G"], dt), Uf), dt, "grad coeff")
+    assert_close(host64(Gp, dt), oracle.grad_project_full(f64(t["G"], dt), Uf), dt, "grad full")
+    W0 = synth.projection_weight(640, wl.d, seed=2, dtype=dt)
+    W = to_device(W0, dt)
+    codec.weight_reproject_list([W], "right")
+    assert_close(host64(W, dt), oracle.weight_reproject(f64(W0, dt), Uf, "right"), dt, "reproject")
+    assert codec.take_status() == 0
