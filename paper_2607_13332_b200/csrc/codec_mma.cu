@@ -200,7 +200,7 @@ cudaError_t launch_umma_one(const MmaArgs &a, const UmmaMaps &maps, int sm_count
   }
   // pairs of CTAs (clusters of two) that share their odd tile; see the kernel's schedule
   const int64_t ntiles = (a.n + kUmmaTile - 1) / kUmmaTile;
-  int64_t pairs = (ntiles + 1) / 2;
+  int64_t pairs = ntiles;   // with few tiles every pair has one and splits it over d
   if (pairs > sm_count / 2) pairs = sm_count / 2;
   if (pairs < 1) {   // a single SM: plain launch
     kernel<<<(unsigned)(ntiles < sm_count ? ntiles : sm_count), kUmmaThreads, smem, stream>>>(a, maps);
