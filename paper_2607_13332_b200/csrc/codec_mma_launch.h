@@ -23,7 +23,11 @@ struct MmaArgs {
 // Shapes the tensor-core kernels take (alignment is checked by the caller).
 bool codec_mma_supports(int d, int k);
 
-// Project-then-expand of up to 8 matrices in ONE launch of the tcgen05 kernel (a.U, a.ldu, a.d,
+// Most matrices one launch of the fused project-then-expand kernel takes (its tensor maps travel
+// as kernel parameters: 2 x 128 bytes per matrix).
+constexpr int kMaxFusedMatrices = 32;
+
+// Project-then-expand of up to kMaxFusedMatrices matrices in ONE launch of the tcgen05 kernel (a.U, a.ldu, a.d,
 // a.k are read from `a`): [rows[i] x d] with the subspace on the columns, or, with `left`,
 // [d x rows[i]] with the subspace on the rows.  cudaErrorNotSupported when the shapes or
 // alignments are not the kernel's, and nothing has been launched then.

@@ -31,6 +31,7 @@
 // (when the caller gave a status word) and the kernel still runs to its end.
 #pragma once
 
+#include "codec_mma_launch.h"
 #include "codec_umma.cuh"
 
 namespace ssn {
@@ -81,7 +82,7 @@ struct UmmaRoundTripConfig {
   static constexpr int kSmemBytes = 1024 + kStagesN * kStageBytes + kFixedBytes + kBars * 8 + 16;
 };
 
-constexpr int kRoundTripMaxMatrices = 8;
+constexpr int kRoundTripMaxMatrices = kMaxFusedMatrices;
 
 // One launch takes up to kRoundTripMaxMatrices matrices [rows_i x d] (the output projections of
 // a block, say): the tiles of all of them are dealt to the CTAs as one list.

@@ -141,14 +141,14 @@ ssn_status_t launch_token_kernel(const TokenArgs &a, int32_t dtype, cudaStream_t
 
 namespace ssn {
 namespace {
-// RIGHT re-projection of `count` matrices [rows[i] x d]: groups of up to 8 go to the fused
+// RIGHT re-projection of `count` matrices [rows[i] x d]: groups of up to kMaxFusedMatrices go to the fused
 // tcgen05 kernel in one launch each; what that kernel does not take goes matrix by matrix.
 ssn_status_t reproject_right_list(const ssn_codec_t *codec, void *const *W_ptrs, const int64_t *rows,
                                   const int64_t *ldw, int32_t count, cudaStream_t s) {
   const int sms = sm_count_of_current_device();
   int32_t done = 0;
   while (done < count) {
-    const int32_t take = count - done < 8 ? count - done : 8;
+    const int32_t take = count - done < kMaxFusedMatrices ? count - done : kMaxFusedMatrices;
     bool fused = false;
     if (codec->dtype == SSN_BF16 && sms > 0 && aligned16(codec->U) && (codec->ldu & 7) == 0) {
       MmaArgs m{};
@@ -156,8 +156,8 @@ ssn_status_t reproject_right_list(const ssn_codec_t *codec, void *const *W_ptrs,
       m.ldu = codec->ldu;
       m.d = codec->d;
       m.k = codec->k;
-      const __nv_bfloat16 *src[8];
-      __nv_bfloat16 *dst[8];
+      const __nv_bfloat16 *src[kMaxFusedMatrices];
+      __nv_bfloat16 *dst[kMaxFusedMatrices];
       for (int32_t i = 0; i < take; ++i) src[i] = dst[i] = static_cast<__nv_bfloat16 *>(W_ptrs[done + i]);
       cudaError_t e = launch_codec_umma_roundtrip_list(m, src, dst, rows + done, ldw + done, ldw + done, take,
                                                        sms, s, false);
@@ -194,7 +194,7 @@ ssn_status_t reproject_right_list(const ssn_codec_t *codec, void *const *W_ptrs,
 
 namespace ssn {
 namespace {
-// LEFT re-projection of up to 8 weights [d x cols[i]] on the fused tcgen05 kernel; false when
+// LEFT re-projection of up to kMaxFusedMatrices weights [d x cols[i]] on the fused tcgen05 kernel; false when
 // that kernel does not take the call (nothing launched).
 bool try_reproject_left_fused(const ssn_codec_t *codec, void *const *W_ptrs, const int64_t *cols,
                               const int64_t *ldw, int32_t count, cudaStream_t s, ssn_status_t *st) {
@@ -206,8 +206,8 @@ bool try_reproject_left_fused(const ssn_codec_t *codec, void *const *W_ptrs, con
   m.ldu = codec->ldu;
   m.d = codec->d;
   m.k = codec->k;
-  const __nv_bfloat16 *src[8];
-  __nv_bfloat16 *dst[8];
+  const __nv_bfloat16 *src[kMaxFusedMatrices];
+  __nv_bfloat16 *dst[kMaxFusedMatrices];
   for (int32_t i = 0; i < count; ++i) src[i] = dst[i] = static_cast<__nv_bfloat16 *>(W_ptrs[i]);
   cudaError_t e = launch_codec_umma_roundtrip_list(m, src, dst, cols, ldw, ldw, count, sms, s, true);
   if (e == cudaErrorNotSupported) return false;
@@ -246,14 +246,14 @@ ssn_status_t reproject_left_general(const ssn_codec_t *codec, void *W, int64_t c
   return launch_status(2);
 }
 
-// LEFT re-projection of `count` weights [d x cols[i]]: groups of up to 8 on the fused kernel, the
+// LEFT re-projection of `count` weights [d x cols[i]]: groups of up to kMaxFusedMatrices on the fused kernel, the
 // rest one by one through the workspace.
 ssn_status_t reproject_left_list(const ssn_codec_t *codec, void *const *W_ptrs, const int64_t *cols,
                                  const int64_t *ldw, int32_t count, void *workspace,
                                  size_t workspace_bytes, cudaStream_t s) {
   int32_t done = 0;
   while (done < count) {
-    const int32_t take = count - done < 8 ? count - done : 8;
+    const int32_t take = count - done < kMaxFusedMatrices ? count - done : kMaxFusedMatrices;
     ssn_status_t st;
     if (try_reproject_left_fused(codec, W_ptrs + done, cols + done, ldw + done, take, s, &st)) {
       if (st != SSN_OK) return st;

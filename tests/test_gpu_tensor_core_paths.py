@@ -158,7 +158,7 @@ def test_reproject_rows_list_of_unequal_weights():
     U0 = synth.to_storage(synth.subspace_basis(d, k, seed=3), dt)
     codec = Codec(dt, to_device(U0, dt))
     U = f64(U0, dt)
-    rows = [640, 130, 1, 1024, 77, 256, 300, 128, 999, 64]      # more than one launch's worth
+    rows = [640, 130, 1, 1024, 77, 256, 300, 128, 999, 64] + [96, 160, 33] * 9      # 37: more than one launch's worth
     W0s = [synth.to_storage(np.random.default_rng(r).standard_normal((r, d)) * 0.05, dt) for r in rows]
     views = [padded(r, d, d + 8 * (i % 3), dt, fill=to_device(w, dt)) for i, (r, w) in enumerate(zip(rows, W0s))]
     codec.weight_reproject_rows([v for v, _ in views])
