@@ -218,7 +218,13 @@ cudaError_t launch_umma_one(const MmaArgs &a, const UmmaMaps &maps, int sm_count
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, kernel, a, maps);
+  cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, a, maps);
+  if (e == cudaSuccess) return e;
+  // a device that cannot co-schedule the pairs: the same kernel without clusters
+  cudaGetLastError();
+  const int64_t grid = ntiles < sm_count ? ntiles : sm_count;
+  kernel<<<(unsigned)grid, kUmmaThreads, smem, stream>>>(a, maps);
+  return cudaGetLastError();
 }
 
 template <int NTP>
