@@ -254,6 +254,8 @@ cudaError_t launch_codec_umma_project(const MmaArgs &a, bool shift, int sm_count
   const int ntp = 2 * ((a.k + 15) / 16);
   MmaArgs b = a;
   if (!shift) b.shift.EU = b.shift.PU = nullptr;
+  // whole sequences of 128-position blocks: tiles of one block share their positional product
+  b.pshare = has_e && has_p && a.k <= 64 && a.n % a.shift.seq_len == 0 ? 1 : 0;
   UmmaMaps maps;
   if (!make_sw128_map(&maps.x, a.src, a.n, a.d, a.lds, kUmmaTile)) return cudaErrorNotSupported;
   if (!make_sw128_map(&maps.u, a.U, a.d, a.k, a.ldu, kUmmaCols)) return cudaErrorNotSupported;

@@ -17,6 +17,7 @@ struct MmaArgs {
   int64_t lds, ldzin, ldzout, lddst, ldu;
   int64_t n;
   int32_t d, k;
+  int32_t pshare;             // projection kernel: the batch is whole sequences, share P U per block
   ShiftTables shift;
 };
 

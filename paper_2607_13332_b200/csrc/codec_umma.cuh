@@ -152,8 +152,10 @@ struct UmmaProjectConfig {
   static constexpr int kAccCols = kN <= 32 ? 32 : (kN <= 64 ? 64 : 128);   // TMEM columns per accumulator
   static constexpr int kIssuers = kATiles;                          // one MMA-issuing thread per A operand
   static constexpr int kBufs = 2 * kIssuers * kAccCols <= 512 ? 2 : 1;   // accumulator sets (tiles in flight)
-  static constexpr int kTmemCols = (kBufs * kIssuers * kAccCols) <= 128 ? 128 : ((kBufs * kIssuers * kAccCols) <= 256 ? 256 : 512);
-  static_assert(kBufs * kIssuers * kAccCols <= 512, "accumulators do not fit in tensor memory");
+  // accumulator slots; with E and P and N <= 64 one more holds the shared positional product
+  static constexpr int kAccSlots = kBufs * kIssuers + ((HAS_E && HAS_P && kN <= 64) ? 1 : 0);
+  static constexpr int kTmemCols = (kAccSlots * kAccCols) <= 128 ? 128 : ((kAccSlots * kAccCols) <= 256 ? 256 : 512);
+  static_assert(kAccSlots * kAccCols <= 512, "accumulators do not fit in tensor memory");
   static constexpr int kBarBytes = (2 * kStagesN + 6) * 8 + 16;
   static constexpr int kSmemBytes = 1024 + kStagesN * kStageBytes + kBarBytes;
 };
@@ -200,19 +202,54 @@ codec_umma_project_kernel(const MmaArgs a, const __grid_constant__ UmmaMaps maps
   asm volatile("mov.u32 %0, %%cluster_nctaid.x;\n" : "=r"(cluster_size));
   asm volatile("mov.u32 %0, %%cluster_ctarank;\n" : "=r"(cta_rank));
   const int64_t pairs = gridDim.x / cluster_size, pair = blockIdx.x / cluster_size;
-  const int64_t pair_tiles = pair < ntiles ? (ntiles - pair + pairs - 1) / pairs : 0;
+  // Sharing the positional product.  Tiles at the same 128-position block of different sequences
+  // subtract the same P U.  When the batch is made of whole sequences (a.pshare), the tiles are
+  // enumerated position-block-major (L = block * sequences + sequence), every pair takes a
+  // contiguous range of L, and a CTA keeps P U of its current block in a persistent accumulator:
+  // the P rows are loaded and contracted only when the block changes.
+  constexpr bool kCanShare = HAS_E && HAS_P && Cfg::kN <= 64;
+  const bool pshare = kCanShare && a.pshare != 0;
+  const int64_t nseq = pshare ? a.n / a.shift.seq_len : 1;
+  const int64_t nblk = pshare ? a.shift.seq_len / kUmmaTile : 1;
+  const int64_t l_lo = pshare ? (ntiles * pair) / pairs : 0;
+  const int64_t pair_tiles = pshare ? (ntiles * (pair + 1)) / pairs - l_lo
+                                    : (pair < ntiles ? (ntiles - pair + pairs - 1) / pairs : 0);
   const bool has_split = cluster_size == 2 && (pair_tiles & 1) && nstage >= 2;
   const int my_tiles = (int)(cluster_size == 2
                                  ? pair_tiles / 2 + (((pair_tiles & 1) && (has_split || cta_rank == 0)) ? 1 : 0)
                                  : pair_tiles);
   // i-th tile of this CTA: index, stage range, whether it is the split one
+  auto block_of = [&](int64_t j) { return (l_lo + j) / nseq; };   // position block of the pair's j-th tile
   auto schedule = [&](int i, int64_t &tile, int &st_lo, int &st_hi, bool &split) {
     split = has_split && i == my_tiles - 1;
     const int64_t j = cluster_size == 2 ? (split ? pair_tiles - 1 : 2 * (int64_t)i + cta_rank) : i;
-    tile = pair + j * pairs;
+    if (pshare) {
+      const int64_t L = l_lo + j, blk = L / nseq;
+      tile = (L - blk * nseq) * nblk + blk;
+    } else {
+      tile = pair + j * pairs;
+    }
     st_lo = split && cta_rank == 1 ? nstage / 2 : 0;
     st_hi = split && cta_rank == 0 ? nstage / 2 : nstage;
   };
+  // What this CTA does about P U on its i-th tile, given the block it has cached (-1: none):
+  // 0 = load and contract the P rows over its stage range, 1 = use the cached product,
+  // 2 = nothing (rank 1 on the split tile when rank 0 subtracts its cached full product).
+  auto p_action = [&](int i, bool split, int64_t &cached_blk) {
+    if (!pshare) return 0;
+    const int64_t j = cluster_size == 2 ? (split ? pair_tiles - 1 : 2 * (int64_t)i + cta_rank) : i;
+    const int64_t blk = block_of(j);
+    if (!split) {
+      if (cached_blk == blk) return 1;
+      cached_blk = blk;
+      return 0;
+    }
+    // rank 0 reaches the split tile with the block of its previous tile (j - 2) cached
+    const bool rank0_has = pair_tiles >= 3 && block_of(pair_tiles - 3) == blk;
+    cached_blk = -1;
+    return rank0_has ? (cta_rank == 0 ? 1 : 2) : 0;
+  };
+  constexpr int kPersistentAcc = 2 * Cfg::kIssuers;   // TMEM slot (of kAccCols columns) of the cached P U
 
   if (threadIdx.x == 0) {
     mbar_init(partial_ready_bar, 128);
@@ -248,6 +285,7 @@ codec_umma_project_kernel(const MmaArgs a, const __grid_constant__ UmmaMaps maps
     // ------------------------------------------------------------------------- producer
     int slot = 0;
     uint32_t parity = 1;   // a fresh "empty" barrier passes a wait on parity 1
+    int64_t cached_blk = -1;
     for (int it = 0; it < my_tiles; ++it) {
       int64_t tile;
       int st_lo, st_hi;
@@ -255,14 +293,15 @@ codec_umma_project_kernel(const MmaArgs a, const __grid_constant__ UmmaMaps maps
       schedule(it, tile, st_lo, st_hi, split);
       const int64_t tok0 = tile * kUmmaTile;
       const int pos0 = HAS_P ? (int)(tok0 % a.shift.seq_len) : 0;
+      const bool load_p = HAS_P && p_action(it, split, cached_blk) == 0;
       for (int st = st_lo; st < st_hi; ++st) {
         if (!dead && !mbar_wait(empty_bar(slot), parity)) timed_out();
         const uint32_t base = smem0 + (uint32_t)slot * Cfg::kStageBytes;
         const uint32_t bar = full_bar(slot);
         if (lane == 0) {
-          mbar_expect_tx(bar, Cfg::kTmaBytes);
+          mbar_expect_tx(bar, Cfg::kTmaBytes - (HAS_P && !load_p ? Cfg::kATileBytes : 0));
           tma_load_2d(base, &maps.x, bar, st * kUmmaCols, (int)tok0);
-          if (HAS_P) tma_load_2d(base + kPTile * Cfg::kATileBytes, &maps.p, bar, st * kUmmaCols, pos0);
+          if (load_p) tma_load_2d(base + kPTile * Cfg::kATileBytes, &maps.p, bar, st * kUmmaCols, pos0);
 #pragma unroll
           for (int ug = 0; ug < Cfg::kUGroups; ++ug)
             tma_load_2d(base + Cfg::kATiles * Cfg::kATileBytes + ug * Cfg::kUGroupBytes,
@@ -290,6 +329,8 @@ codec_umma_project_kernel(const MmaArgs a, const __grid_constant__ UmmaMaps maps
       int slot = 0;
       uint32_t parity = 0;
       int64_t tcount = 0;
+      int64_t cached_blk = -1;
+      const bool p_issuer = HAS_P && which == kPTile;
       for (int it = 0; it < my_tiles; ++it, ++tcount) {
         int64_t tile;
         int st_lo, st_hi;
@@ -298,8 +339,17 @@ codec_umma_project_kernel(const MmaArgs a, const __grid_constant__ UmmaMaps maps
         const int buf = (int)(tcount % Cfg::kBufs);
         const uint32_t acc_parity = (uint32_t)((tcount / Cfg::kBufs) & 1);
         if (!dead && !mbar_wait(acc_empty_bar(buf), acc_parity ^ 1u)) timed_out();
+        // the P issuer of a sharing launch: contract only when the block changes, into the
+        // persistent accumulator, once the previous tile's epilogue has read the old product
+        const bool contract = !(p_issuer && p_action(it, split, cached_blk) != 0);
+        if (p_issuer && pshare && contract && tcount > 0) {
+          const int64_t prev = tcount - 1;
+          if (!dead && !mbar_wait(acc_empty_bar((int)(prev % Cfg::kBufs)), (uint32_t)((prev / Cfg::kBufs) & 1)))
+            timed_out();
+        }
         asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
-        const uint32_t d_tmem = tmem_base + (uint32_t)(buf * Cfg::kIssuers + which) * Cfg::kAccCols;
+        const uint32_t d_tmem =
+            tmem_base + (uint32_t)(p_issuer && pshare ? kPersistentAcc : buf * Cfg::kIssuers + which) * Cfg::kAccCols;
         for (int st = st_lo; st < st_hi; ++st) {
           if (!dead && !mbar_wait(full_bar(slot), parity)) timed_out();
           asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
@@ -308,9 +358,11 @@ codec_umma_project_kernel(const MmaArgs a, const __grid_constant__ UmmaMaps maps
           // is 32 bytes of an A row and 16 rows = 2048 bytes of the U slice
           const uint64_t adesc = adesc0 + umma_desc_addr(base + (uint32_t)which * Cfg::kATileBytes);
           const uint64_t bdesc = bdesc0 + umma_desc_addr(base + Cfg::kATiles * Cfg::kATileBytes);
+          if (contract) {
 #pragma unroll
-          for (int j = 0; j < kUmmaCols / 16; ++j)
-            umma_bf16(d_tmem, adesc + j * 2, bdesc + j * 128, idesc, (st > st_lo || j > 0) ? 1u : 0u);
+            for (int j = 0; j < kUmmaCols / 16; ++j)
+              umma_bf16(d_tmem, adesc + j * 2, bdesc + j * 128, idesc, (st > st_lo || j > 0) ? 1u : 0u);
+          }
           umma_commit(empty_bar(slot));
           if (st == st_hi - 1) umma_commit(acc_full_bar(buf));
           if (++slot == S) {
@@ -375,12 +427,14 @@ codec_umma_project_kernel(const MmaArgs a, const __grid_constant__ UmmaMaps maps
     // ------------------------------------------------------------------------- epilogue
     const int quarter = warp & 3;   // the TMEM lanes this warp may read: 32*quarter .. +31
     int64_t tcount = 0;
+    int64_t cached_blk = -1;
     const bool vec = ((a.ldzout & 7) == 0) && ((reinterpret_cast<uintptr_t>(a.zout) & 15) == 0);
     for (int it = 0; it < my_tiles; ++it, ++tcount) {
       int64_t tile;
       int st_lo, st_hi;
       bool split;
       schedule(it, tile, st_lo, st_hi, split);
+      const int p_act = HAS_P ? p_action(it, split, cached_blk) : 0;
       const int buf = (int)(tcount % Cfg::kBufs);
       const uint32_t acc_parity = (uint32_t)((tcount / Cfg::kBufs) & 1);
       if (!dead && !mbar_wait(acc_full_bar(buf), acc_parity)) timed_out();
@@ -393,10 +447,16 @@ codec_umma_project_kernel(const MmaArgs a, const __grid_constant__ UmmaMaps maps
       asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
 #pragma unroll
       for (int op = 1; op < Cfg::kIssuers; ++op) {   // Z = X.U - E.U - P.U
+        const bool is_p = HAS_P && op == kPTile;
+        if (is_p && p_act == 2) continue;              // the peer subtracts the whole product
+        // a sharing launch keeps P.U in its persistent accumulator
+        const uint32_t oaddr = is_p && pshare
+                                   ? tmem_base + ((uint32_t)(quarter * 32) << 16) + kPersistentAcc * Cfg::kAccCols
+                                   : taddr + op * Cfg::kAccCols;
 #pragma unroll
         for (int q = 0; q < Cfg::kN / 16; ++q) {
           uint32_t w[16];
-          tmem_ld16(taddr + op * Cfg::kAccCols + q * 16, w);
+          tmem_ld16(oaddr + q * 16, w);
           asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
 #pragma unroll
           for (int i = 0; i < 16; ++i) v[q][i] = __float_as_uint(__uint_as_float(v[q][i]) - __uint_as_float(w[i]));
