@@ -171,11 +171,11 @@ bool make_sw128_map3(CUtensorMap *map, const void *base, int64_t cols, int64_t n
             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <bool HAS_E, bool HAS_P>
+template <int KG, bool HAS_E, bool HAS_P>
 cudaError_t launch_umma_expand_one(const MmaArgs &a, const ExpandGeometry &geo, const UmmaExpandMaps &maps,
                                    int sm_count, cudaStream_t stream) {
-  auto kernel = codec_umma_expand_kernel<HAS_E, HAS_P>;
-  constexpr int smem = UmmaExpandConfig<HAS_E, HAS_P>::kSmemBytes;
+  auto kernel = codec_umma_expand_kernel<KG, HAS_E, HAS_P>;
+  constexpr int smem = UmmaExpandConfig<KG, HAS_E, HAS_P>::kSmemBytes;
   static bool configured = false;
   if (!configured) {
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
@@ -355,12 +355,12 @@ cudaError_t launch_codec_umma_roundtrip(const MmaArgs &a, int sm_count, cudaStre
 }
 
 // Expansion (decompress) on tcgen05.  Returns cudaErrorNotSupported when the call should take the
-// mma.sync kernel instead: k > 64, d not a multiple of 128, few tokens, no tensor map, or a
+// mma.sync kernel instead: k > 128, d not a multiple of 128, few tokens, no tensor map, or a
 // position table with explicit positions / a batch that is not made of groups of 8 whole
 // sequences whose length is a multiple of 16.
 cudaError_t launch_codec_umma_expand(const MmaArgs &a, bool shift, int sm_count, cudaStream_t stream) {
   if (a.zin == nullptr || a.dst == nullptr || a.src != nullptr) return cudaErrorNotSupported;
-  if (a.d % kChunkCols != 0 || a.k > 64 || a.n < 4 * kUmmaTile || a.n > 0x7fffffffLL)
+  if (a.d % kChunkCols != 0 || a.k > 128 || a.n < 4 * kUmmaTile || a.n > 0x7fffffffLL)
     return cudaErrorNotSupported;
   const bool has_e = shift && a.shift.E != nullptr, has_p = shift && a.shift.P != nullptr;
   ExpandGeometry geo{};
@@ -395,11 +395,17 @@ cudaError_t launch_codec_umma_expand(const MmaArgs &a, bool shift, int sm_count,
     maps.p = maps.z;
   }
   if (!make_sw128_map(&maps.u, a.U, a.d, a.k, a.ldu, kUmmaCols)) return cudaErrorNotSupported;
-  if (!make_sw128_map(&maps.u_wide, a.U, a.d, 64, a.ldu, kUmmaCols)) return cudaErrorNotSupported;
-  if (has_e && has_p) return launch_umma_expand_one<true, true>(a, geo, maps, sm_count, stream);
-  if (has_e) return launch_umma_expand_one<true, false>(a, geo, maps, sm_count, stream);
-  if (has_p) return launch_umma_expand_one<false, true>(a, geo, maps, sm_count, stream);
-  return launch_umma_expand_one<false, false>(a, geo, maps, sm_count, stream);
+  if (!make_sw128_map(&maps.u_wide, a.U, a.d, a.k <= 64 ? 64 : 128, a.ldu, kUmmaCols)) return cudaErrorNotSupported;
+  if (a.k > 64) {
+    if (has_e && has_p) return launch_umma_expand_one<2, true, true>(a, geo, maps, sm_count, stream);
+    if (has_e) return launch_umma_expand_one<2, true, false>(a, geo, maps, sm_count, stream);
+    if (has_p) return launch_umma_expand_one<2, false, true>(a, geo, maps, sm_count, stream);
+    return launch_umma_expand_one<2, false, false>(a, geo, maps, sm_count, stream);
+  }
+  if (has_e && has_p) return launch_umma_expand_one<1, true, true>(a, geo, maps, sm_count, stream);
+  if (has_e) return launch_umma_expand_one<1, true, false>(a, geo, maps, sm_count, stream);
+  if (has_p) return launch_umma_expand_one<1, false, true>(a, geo, maps, sm_count, stream);
+  return launch_umma_expand_one<1, false, false>(a, geo, maps, sm_count, stream);
 }
 
 bool codec_mma_supports(int d, int k) {

@@ -1,4 +1,5 @@
-// tcgen05 / TMA expansion kernel of the SSN codec (bf16, sm_100a), k <= 64:
+// tcgen05 / TMA expansion kernel of the SSN codec (bf16, sm_100a), k <= 128 (KG = 1 or 2 groups
+// of 64 coordinates, each a 128-byte operand row):
 //     Xhat = Z U^T + E[ids] + P[pos]          decompress (receiver side of Eq. ssn_compress)
 //
 // A tile is 128 tokens, a chunk 128 output columns accumulated in 128 TMEM columns:
@@ -44,19 +45,20 @@ __device__ __forceinline__ void tma_store_3d(const CUtensorMap *map, uint32_t sr
                ::"l"(map), "r"(src), "r"(c0), "r"(c1), "r"(c2) : "memory");
 }
 
-template <bool HAS_E, bool HAS_P>
+template <int KG, bool HAS_E, bool HAS_P>
 struct UmmaExpandConfig {
   static constexpr int kTileBytes = kUmmaTile * 128;            // [128 rows x 128 B]
-  static constexpr int kU2Bytes = kChunkCols * 128;             // 128 rows of U, K-major
+  static constexpr int kZBytes = KG * kTileBytes;               // one Z tile: KG groups of 64 coordinates
+  static constexpr int kU2Bytes = KG * kChunkCols * 128;        // 128 rows of U, K-major, KG groups
   static constexpr int kPBytes = HAS_P ? 2 * kGridPos * 128 : 0;   // 16 rows of P, two 64-column groups
   static constexpr int kUStageBytes = kU2Bytes + kPBytes;
-  static constexpr int kUStages = HAS_E ? 2 : 3;   // with E the shared memory is better spent on its ring
+  static constexpr int kUStages = (HAS_E || KG == 2) ? 2 : 3;   // with E the shared memory is better spent on its ring
   static constexpr int kEStageBytes = kTileBytes;               // E rows of 64 columns of a chunk
   // Without E the epilogue warps stage their output in two [32 x 128 B] slabs each; with E the
   // sum is formed in place in the E stage, which is then the source of the TMA store.
   static constexpr int kStagingBytes = HAS_E ? 0 : 8 * 2 * 4096;
   static constexpr int kFixedBytes =
-      2 * kTileBytes + (HAS_P ? kTileBytes : 0) + kUStages * kUStageBytes + kStagingBytes;
+      2 * kZBytes + (HAS_P ? kTileBytes : 0) + kUStages * kUStageBytes + kStagingBytes;
   static constexpr int kMaxSmem = 227 * 1024;
   static constexpr int kEFit = (kMaxSmem - 1024 - 512 - kFixedBytes) / kEStageBytes;
   static constexpr int kEStages = HAS_E ? (kEFit < 8 ? kEFit : 8) : 0;
@@ -80,10 +82,10 @@ struct ExpandGeometry {
   int64_t ntiles;
 };
 
-template <bool HAS_E, bool HAS_P>
+template <int KG, bool HAS_E, bool HAS_P>
 __global__ void __launch_bounds__(kExpandThreads, 1)
 codec_umma_expand_kernel(const MmaArgs a, const ExpandGeometry geo, const __grid_constant__ UmmaExpandMaps maps) {
-  using Cfg = UmmaExpandConfig<HAS_E, HAS_P>;
+  using Cfg = UmmaExpandConfig<KG, HAS_E, HAS_P>;
   constexpr int SU = Cfg::kUStages, SE = Cfg::SE;
   extern __shared__ __align__(128) unsigned char smem_raw[];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -93,7 +95,7 @@ codec_umma_expand_kernel(const MmaArgs a, const ExpandGeometry geo, const __grid
 
   const uint32_t smem0 = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t z_base = smem0;                                         // two Z tiles
-  const uint32_t sel = z_base + 2 * Cfg::kTileBytes;                     // selection matrix (HAS_P)
+  const uint32_t sel = z_base + 2 * Cfg::kZBytes;                        // selection matrix (HAS_P)
   const uint32_t u_ring = sel + (HAS_P ? Cfg::kTileBytes : 0);
   const uint32_t staging = u_ring + SU * Cfg::kUStageBytes;
   const uint32_t e_ring = staging + Cfg::kStagingBytes;
@@ -191,8 +193,10 @@ codec_umma_expand_kernel(const MmaArgs a, const ExpandGeometry geo, const __grid
       const int zb = (int)(tcount & 1);
       if (!dead && !mbar_wait(z_empty_bar(zb), (uint32_t)(((tcount >> 1) & 1) ^ 1))) timed_out();
       if (lane == 0) {
-        mbar_expect_tx(z_full_bar(zb), Cfg::kTileBytes);
-        tma_load_3d(z_base + zb * Cfg::kTileBytes, &maps.z, z_full_bar(zb), 0, c1, c2);
+        mbar_expect_tx(z_full_bar(zb), Cfg::kZBytes);
+#pragma unroll
+        for (int kg = 0; kg < KG; ++kg)
+          tma_load_3d(z_base + zb * Cfg::kZBytes + kg * Cfg::kTileBytes, &maps.z, z_full_bar(zb), kg * 64, c1, c2);
       }
       int q0, q1;
       chunk_range(tile, q0, q1);
@@ -201,9 +205,12 @@ codec_umma_expand_kernel(const MmaArgs a, const ExpandGeometry geo, const __grid
         const uint32_t base = u_ring + (uint32_t)slot * Cfg::kUStageBytes;
         if (lane == 0) {
           mbar_expect_tx(u_full_bar(slot), Cfg::kUStageBytes);
-          tma_load_2d(base, &maps.u_wide, u_full_bar(slot), 0, q * kChunkCols);
-          tma_load_2d(base + 8192, q == nchunks - 1 ? &maps.u : &maps.u_wide, u_full_bar(slot), 0,
-                      q * kChunkCols + 64);
+#pragma unroll
+          for (int kg = 0; kg < KG; ++kg) {   // per group of 64 coordinates: 128 rows of 128 bytes
+            tma_load_2d(base + kg * Cfg::kTileBytes, &maps.u_wide, u_full_bar(slot), kg * 64, q * kChunkCols);
+            tma_load_2d(base + kg * Cfg::kTileBytes + 8192, q == nchunks - 1 ? &maps.u : &maps.u_wide,
+                        u_full_bar(slot), kg * 64, q * kChunkCols + 64);
+          }
           if (HAS_P) {
             tma_load_2d(base + Cfg::kU2Bytes, &maps.p, u_full_bar(slot), q * kChunkCols, c1);
             tma_load_2d(base + Cfg::kU2Bytes + kGridPos * 128, &maps.p, u_full_bar(slot), q * kChunkCols + 64, c1);
@@ -230,7 +237,7 @@ codec_umma_expand_kernel(const MmaArgs a, const ExpandGeometry geo, const __grid
       for (int64_t tile = tile_lo; tile <= tile_hi; ++tile, ++tcount) {
         const int zb = (int)(tcount & 1);
         if (!dead && !mbar_wait(z_full_bar(zb), (uint32_t)((tcount >> 1) & 1))) timed_out();
-        const uint64_t zd = kdesc + umma_desc_addr(z_base + zb * Cfg::kTileBytes);
+        const uint64_t zd = kdesc + umma_desc_addr(z_base + zb * Cfg::kZBytes);
         int q0, q1;
         chunk_range(tile, q0, q1);
         for (int q = q0; q < q1; ++q, ++ccount) {
@@ -241,7 +248,10 @@ codec_umma_expand_kernel(const MmaArgs a, const ExpandGeometry geo, const __grid
           const uint32_t base = u_ring + (uint32_t)slot * Cfg::kUStageBytes;
           const uint32_t dacc = tmem_base + (uint32_t)db * kChunkCols;
           const uint64_t bd = kdesc + umma_desc_addr(base);
-          for (int j = 0; j < ksteps; ++j) umma_bf16(dacc, zd + j * 2, bd + j * 2, idesc_kk, j > 0 ? 1u : 0u);
+          for (int j = 0; j < ksteps; ++j) {   // K step j: 32 bytes into the rows of group j / 4
+            const uint32_t ko = (uint32_t)(j >> 2) * (Cfg::kTileBytes >> 4) + (uint32_t)(j & 3) * 2;
+            umma_bf16(dacc, zd + ko, bd + ko, idesc_kk, j > 0 ? 1u : 0u);
+          }
           if (HAS_P) umma_bf16(dacc, seld, pdesc + umma_desc_addr(base + Cfg::kU2Bytes), idesc_kmn, 1u);
           umma_commit(u_empty_bar(slot));
           umma_commit(d_full_bar(db));

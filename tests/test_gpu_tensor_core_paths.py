@@ -29,6 +29,9 @@ SHAPES = [
     (12, 256, 2048, 128, 999),   # k = 128: two column groups of U; 24 tiles on 12 CTA pairs
     (17, 128, 1024, 96, 500),    # 17 tiles: the last pair splits its tile over d
     (1, 640, 512, 40, 200),      # 5 tiles on 3 pairs, one of them split
+    (16, 128, 1024, 96, 500),    # 64 < k <= 128 on the expansion kernel, 8 x 16 tiles
+    (8, 256, 512, 128, 300),
+    (24, 64, 256, 72, 100),
 ]
 
 
