@@ -352,6 +352,15 @@ codec_umma_expand_kernel(const MmaArgs a, const ExpandGeometry geo, const __grid
             slab = slab0 + (uint32_t)g * 4096;
           }
           const uint32_t srow = slab + lane * 128;
+          // all eight E pieces of the row first, so that their latencies overlap
+          uint32_t e[8][4];
+          if (HAS_E) {
+#pragma unroll
+            for (int c = 0; c < 8; ++c)
+              asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];\n"
+                           : "=r"(e[c][0]), "=r"(e[c][1]), "=r"(e[c][2]), "=r"(e[c][3])
+                           : "r"(srow + ((c ^ (lane & 7)) << 4)));
+          }
 #pragma unroll
           for (int c = 0; c < 8; ++c) {
             const uint32_t *w = &v[c >> 1][(c & 1) * 8];
@@ -360,17 +369,11 @@ codec_umma_expand_kernel(const MmaArgs a, const ExpandGeometry geo, const __grid
 #pragma unroll
             for (int i = 0; i < 8; ++i) f[i] = __uint_as_float(w[i]);
             if (HAS_E) {   // the sum replaces the E piece
-              uint32_t e0, e1, e2, e3;
-              asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];\n"
-                           : "=r"(e0), "=r"(e1), "=r"(e2), "=r"(e3) : "r"(addr));
-              f[0] += __uint_as_float(e0 << 16);
-              f[1] += __uint_as_float(e0 & 0xFFFF0000u);
-              f[2] += __uint_as_float(e1 << 16);
-              f[3] += __uint_as_float(e1 & 0xFFFF0000u);
-              f[4] += __uint_as_float(e2 << 16);
-              f[5] += __uint_as_float(e2 & 0xFFFF0000u);
-              f[6] += __uint_as_float(e3 << 16);
-              f[7] += __uint_as_float(e3 & 0xFFFF0000u);
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                f[2 * i] += __uint_as_float(e[c][i] << 16);
+                f[2 * i + 1] += __uint_as_float(e[c][i] & 0xFFFF0000u);
+              }
             }
             const uint32_t o0 = pack_bf16(f[0], f[1]), o1 = pack_bf16(f[2], f[3]);
             const uint32_t o2 = pack_bf16(f[4], f[5]), o3 = pack_bf16(f[6], f[7]);
