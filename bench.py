@@ -61,7 +61,7 @@ def parse_args():
                          "the E and P rows (the default step gathers; the table variant is always "
                          "timed beside it as compress_prepared_tables)")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
-    ap.add_argument("--sweep", choices=["compress", "reproject"], default=None,
+    ap.add_argument("--sweep", choices=["compress", "reproject", "reparam"], default=None,
                     help="instead of the step: time the compress sweep (d, k, tokens) or the "
                          "re-projection sweep (k, weight shape, 32 layers); one JSON line per point")
     return ap.parse_args()
@@ -450,6 +450,35 @@ def run_sweep(args):
                     print(json.dumps(out), flush=True)
                     del X, Z, ids
             del E, P
+    elif args.sweep == "reparam":
+        # reparameterized SSN (Eq. reparam): Y = (H Zw) U^T for the block's two output projections,
+        # and the head-stage input with the factored embedding, at the benchmark's token count
+        d, k, n = 4096, 40, 65536
+        U = to_device(synth.to_storage(synth.subspace_basis(d, k, 1), dt), dt)
+        codec = Codec(dt, U)
+        Y = torch.empty((n, d), dtype=torch.bfloat16, device="cuda")
+        for name, m in (("out_proj", 4096), ("down_proj", 14336)):
+            H = torch.randn((n, m), device="cuda", generator=gen).bfloat16()
+            Zw = (torch.randn((m, k), device="cuda", generator=gen) / m ** 0.5).bfloat16()
+            us = timed_us(lambda: codec.reparam_project(H, Zw, out=Y), 5)
+            algo = n * m * 2 + n * d * 2 + (m + d) * k * 2
+            print(json.dumps({"sweep": "reparam", "op": "reparam_project", "weight": name, "tokens": n, "m": m,
+                              "d": d, "k": k, "us": round(us, 1), "GBps": round(algo / us / 1e3, 0),
+                              "frac_of_measured": round(algo / us / 1e3 / peak, 3)}), flush=True)
+            del H, Zw
+        E = (torch.randn((vocab, d), device="cuda", generator=gen) * 0.02).bfloat16()
+        P = to_device(synth.to_storage(synth.sinusoidal_positions(seq, d), dt), dt)
+        Elow = torch.randn((vocab, k), device="cuda", generator=gen).bfloat16()
+        head = Codec(dt, U, E, P)
+        wl = synth.STAGE_8B
+        ids_np = synth.token_ids(wl, 3)
+        ids = torch.from_numpy(ids_np).cuda()
+        us = timed_us(lambda: head.head_embed(Elow, ids, seq_len=seq, out=Y), 5)
+        uniq = int(np.unique(ids_np).size)
+        algo = n * d * 2 + uniq * (d + k) * 2 + seq * d * 2 + n * 4 + d * k * 2
+        print(json.dumps({"sweep": "reparam", "op": "head_embed", "tokens": n, "d": d, "k": k,
+                          "us": round(us, 1), "GBps": round(algo / us / 1e3, 0),
+                          "frac_of_measured": round(algo / us / 1e3 / peak, 3)}), flush=True)
     else:
         d = 4096
         for k in synth.REPROJECT_RANKS:

@@ -195,6 +195,38 @@ ssn_status_t ssn_weight_reproject_list(const ssn_codec_t *codec, void *const *W_
                                        void *stream);
 
 /*
+ * Reparameterized SSN (Eq. reparam): an output projection is stored as its low-dimensional
+ * factor Zw [m x k], W_p = Zw U_k^T, whose rows lie in the subspace by construction, and the
+ * block's output
+ *     Y [n x d] = (H [n x m] Zw) U^T
+ * is formed from the two skinny products without ever materialising W_p (H: the activations the
+ * projection acts on, attention output or MLP inner activation, of width m).
+ *   coords     optional [n x k] output of the coordinates H Zw (storage dtype, ldc >= k), or NULL
+ * The coordinates stay in fp32 between the two products on every path.
+ * H and Y must not overlap.  E and P of the codec are not used.
+ */
+ssn_status_t ssn_reparam_project(const ssn_codec_t *codec, const void *H, int64_t ldh, int64_t m,
+                                 const void *Zw, int64_t ldzw, int64_t n_tokens, void *Y,
+                                 int64_t ldy, void *coords, int64_t ldc, void *stream);
+
+/*
+ * Head-stage input of the reparameterized SSN (Sec. 4.1: the trainable embedding is factored as
+ * T_S = Elow U_k^T "with every projection and the embedding parameterized through U_k"):
+ *     X0[t,:] = E[ids[t],:] + Elow[ids[t],:] U^T + P[pos(t),:]
+ * i.e. ssn_decompress applied to the gathered rows of Elow [vocab x k]; compressing X0 gives
+ * those rows back exactly.
+ *   workspace  device scratch of n * kpad * sizeof(element) bytes, kpad = k rounded up to 8,
+ *              16-byte aligned: the gathered coordinates.
+ * ids, pos, seq_len, dev_status as for ssn_decompress; an id outside the table contributes
+ * neither of its two rows.  Elow rows are used whether or not the codec has E.
+ */
+ssn_status_t ssn_head_embed(const ssn_codec_t *codec, const void *Elow, int64_t ldel,
+                            int64_t vocab_low, const int32_t *ids, const int32_t *pos,
+                            int64_t n_tokens, int32_t seq_len, void *X0, int64_t ldx,
+                            void *workspace, size_t workspace_bytes, int32_t *dev_status,
+                            void *stream);
+
+/*
  * LEFT re-projection of ONE weight, W [d x cols] <- U (U^T W), without a caller workspace.
  * (The paper has no counterpart: this is a packaging variant of ssn_weight_reproject.)
  *

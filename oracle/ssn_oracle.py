@@ -23,7 +23,9 @@ raises a status bit instead of failing; the backward pass sends G U.
 Pins (tests/test_oracle_pins.py): hand-worked example, one-hot basis special case, bit-exact
 gather, isometry at k = d, exact round trip inside the subspace, adjoint and finite-difference
 identities, projector identities, explicit d x d projector, element-by-element loops on tiny
-shapes.  No function here is left unpinned.
+shapes; for the reparameterized forms (Eq. reparam): the materialised weight W_p = Z U^T, its
+membership of the subspace, loops, and the exact recovery of the factored embedding's coordinates
+by compress.  No function here is left unpinned.
 """
 
 from __future__ import annotations
@@ -106,3 +108,23 @@ def weight_reproject(W: np.ndarray, U: np.ndarray, side: str) -> np.ndarray:
     if side == "left":
         return U @ (U.T @ W)
     raise ValueError("side must be 'left' or 'right'")
+
+
+def reparam_project(H: np.ndarray, Zw: np.ndarray, U: np.ndarray) -> np.ndarray:
+    """Eq. reparam: an output projection stored as its factor, W_p = Zw U_k^T.  The block's output
+    Y = H W_p is formed as (H Zw) U_k^T, the k coordinates unrounded in between."""
+    H = np.asarray(H, dtype=np.float64)
+    return (H @ np.asarray(Zw, dtype=np.float64)) @ np.asarray(U, dtype=np.float64).T
+
+
+def head_embed(Elow: np.ndarray, U: np.ndarray, E=None, ids=None, P=None, pos=None):
+    """Head-stage input with the factored trainable embedding T_S = Elow U_k^T (Sec. 4.1):
+    X0[t] = T_fixed[ids[t]] + Elow[ids[t]] U_k^T + PE[pos[t]].  A token whose id is outside Elow
+    contributes no trainable row (and, through decompress, no fixed row).  Returns (X0, status)."""
+    Elow = np.asarray(Elow, dtype=np.float64)
+    ids = np.asarray(ids, dtype=np.int64)
+    ok = (ids >= 0) & (ids < Elow.shape[0])
+    Z = np.zeros((ids.shape[0], Elow.shape[1]), dtype=np.float64)
+    Z[ok] = Elow[ids[ok]]
+    return decompress(Z, U, E, ids, P, pos)
+

@@ -67,6 +67,8 @@ _SIGNATURES = {
                                     _vp, _sz, _vp]),
     "ssn_weight_reproject_left_static": (_i32, [_codec_p, _vp, _i64, _i64, _vp]),
     "ssn_prepare_tables": (_i32, [_codec_p, _vp, _i64, _vp, _i64, _vp]),
+    "ssn_reparam_project": (_i32, [_codec_p, _vp, _i64, _i64, _vp, _i64, _i64, _vp, _i64, _vp, _i64, _vp]),
+    "ssn_head_embed": (_i32, [_codec_p, _vp, _i64, _i64, _vp, _vp, _i64, _i32, _vp, _i64, _vp, _sz, _vp, _vp]),
     "ssn_weight_reproject_list": (_i32, [_codec_p, ctypes.POINTER(_vp), ctypes.POINTER(_i64),
                                          ctypes.POINTER(_i64), _i32, _i32, _vp, _sz, _vp]),
     "ssn_static_scratch_bytes": (_sz, []),
@@ -172,6 +174,23 @@ def ssn_weight_reproject_list(codec: ssn_codec_t, W_ptrs, extent, ldw, side: int
     _check(_lib.ssn_weight_reproject_list(ctypes.byref(codec), (_vp * n)(*W_ptrs), (_i64 * n)(*extent),
                                           (_i64 * n)(*ldw), n, side, workspace or None, workspace_bytes,
                                           stream or None), "ssn_weight_reproject_list")
+
+
+def ssn_reparam_project(codec: ssn_codec_t, H: int, ldh: int, m: int, Zw: int, ldzw: int, n_tokens: int,
+                        Y: int, ldy: int, coords: int = 0, ldc: int = 0, stream: int = 0) -> None:
+    """Y [n x d] = (H [n x m] Zw [m x k]) U^T (Eq. reparam), optionally also the coordinates H Zw."""
+    _check(_lib.ssn_reparam_project(ctypes.byref(codec), H or None, ldh, m, Zw or None, ldzw, n_tokens,
+                                    Y or None, ldy, coords or None, ldc, stream or None),
+           "ssn_reparam_project")
+
+
+def ssn_head_embed(codec: ssn_codec_t, Elow: int, ldel: int, vocab_low: int, ids: int, pos: int,
+                   n_tokens: int, seq_len: int, X0: int, ldx: int, workspace: int, workspace_bytes: int,
+                   dev_status: int = 0, stream: int = 0) -> None:
+    """X0[t] = E[ids[t]] + Elow[ids[t]] U^T + P[pos(t)] (head-stage input of the reparameterized SSN)."""
+    _check(_lib.ssn_head_embed(ctypes.byref(codec), Elow or None, ldel, vocab_low, ids or None, pos or None,
+                               n_tokens, seq_len, X0 or None, ldx, workspace or None, workspace_bytes,
+                               dev_status or None, stream or None), "ssn_head_embed")
 
 
 def ssn_prepare_tables(codec: ssn_codec_t, EU: int, ldeu: int, PU: int, ldpu: int,

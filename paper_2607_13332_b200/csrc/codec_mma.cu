@@ -313,7 +313,8 @@ cudaError_t launch_codec_umma_roundtrip_list(const MmaArgs &a, const __nv_bfloat
       if (!make_sw128_map(&maps.s[i], src[i], a.d, rows[i], lds[i], kUmmaCols)) return cudaErrorNotSupported;
       if (!make_sw128_map(&maps.out[i], dst[i], a.d, rows[i], lddst[i], 32)) return cudaErrorNotSupported;
     } else {
-      if (!make_sw128_map(&maps.s[i], src[i], rows[i], a.d, lds[i], kUmmaTile)) return cudaErrorNotSupported;
+      if (!make_sw128_map(&maps.s[i], src[i], rows[i], a.B1 != nullptr ? a.d1 : a.d, lds[i], kUmmaTile))
+        return cudaErrorNotSupported;
       if (!make_sw128_map(&maps.out[i], dst[i], rows[i], a.d, lddst[i], 32)) return cudaErrorNotSupported;
     }
   }
@@ -328,6 +329,13 @@ cudaError_t launch_codec_umma_roundtrip_list(const MmaArgs &a, const __nv_bfloat
   maps.count = count;
   if (!make_sw128_map(&maps.u, a.U, a.d, a.k, a.ldu, kUmmaCols)) return cudaErrorNotSupported;
   if (!make_sw128_map(&maps.u_wide, a.U, a.d, a.k <= 64 ? 64 : 128, a.ldu, kUmmaCols)) return cudaErrorNotSupported;
+  maps.b1 = maps.u;
+  maps.b1_wide = maps.u_wide;
+  if (a.B1 != nullptr) {
+    if (left || a.d1 < kUmmaCols || a.d1 % kUmmaCols != 0) return cudaErrorNotSupported;
+    if (!make_sw128_map(&maps.b1, a.B1, a.d1, a.k, a.ldb1, kUmmaCols)) return cudaErrorNotSupported;
+    if (!make_sw128_map(&maps.b1_wide, a.B1, a.d1, a.k <= 64 ? 64 : 128, a.ldb1, kUmmaCols)) return cudaErrorNotSupported;
+  }
   MmaArgs b = a;
   if (count > 1 || left) b.zout = nullptr;
   const int ntp = 2 * ((a.k + 15) / 16);

@@ -18,6 +18,11 @@ struct MmaArgs {
   int64_t n;
   int32_t d, k;
   int32_t pshare;             // projection kernel: the batch is whole sequences, share P U per block
+  // project-then-expand with two different factors (Eq. reparam, Y = (H Z) U^T): the rows of src
+  // have d1 columns and are contracted with B1 [d1 x k]; nullptr: B1 = U, d1 = d
+  const __nv_bfloat16 *B1;
+  int64_t ldb1;
+  int32_t d1;
   ShiftTables shift;
 };
 

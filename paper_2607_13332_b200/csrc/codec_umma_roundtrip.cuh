@@ -90,6 +90,7 @@ struct UmmaRoundTripMaps {
   // U: 64 x 64 boxes (u_wide: see UmmaMaps); per matrix, S: boxes of 128 rows x 64 columns,
   // out: 32 rows x 64 columns
   CUtensorMap u, u_wide;
+  CUtensorMap b1, b1_wide;   // the factor of pass 1 when it is not U (see MmaArgs::B1), else copies of u, u_wide
   CUtensorMap s[kRoundTripMaxMatrices], out[kRoundTripMaxMatrices];
   int64_t rows[kRoundTripMaxMatrices];
   int32_t tile_start[kRoundTripMaxMatrices + 1];   // first tile of each matrix; [count] = all tiles
@@ -103,7 +104,7 @@ codec_umma_roundtrip_kernel(const MmaArgs a, const __grid_constant__ UmmaRoundTr
   constexpr int S = Cfg::kStagesN, S2 = Cfg::kU2Stages;
   extern __shared__ __align__(128) unsigned char smem_raw[];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int nstage = a.d / kUmmaCols;
+  const int nstage = (a.B1 != nullptr ? a.d1 : a.d) / kUmmaCols;   // pass 1 runs over the columns of the source
   const int nchunks = a.d / kChunkCols;
   const int64_t ntiles = maps.tile_start[maps.count];
   // tile -> matrix and first row (LEFT: first column)
@@ -183,7 +184,7 @@ codec_umma_roundtrip_kernel(const MmaArgs a, const __grid_constant__ UmmaRoundTr
           }
 #pragma unroll
           for (int ug = 0; ug < Cfg::kKG; ++ug)
-            tma_load_2d(base + Cfg::kTileBytes + ug * Cfg::kUGroupBytes, st == nstage - 1 ? &maps.u : &maps.u_wide,
+            tma_load_2d(base + Cfg::kTileBytes + ug * Cfg::kUGroupBytes, st == nstage - 1 ? &maps.b1 : &maps.b1_wide,
                         full_bar(slot), ug * 64, st * kUmmaCols);
         }
         __syncwarp();

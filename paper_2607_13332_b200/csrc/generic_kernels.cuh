@@ -16,6 +16,9 @@ struct TokenArgs {
   int64_t lds, ldzin, ldzout, lddst, ldu;
   int64_t n;
   int32_t d, k;
+  const void *U2;     // expansion factor [d2 x k] when it differs from U (Eq. reparam), else nullptr
+  int64_t ldu2;
+  int32_t d2;
   int32_t sub_shift;  // phase 1 subtracts E[ids]+P[pos]   (Eq. ssn_compress)
   int32_t add_shift;  // phase 2 adds E[ids]+P[pos] back   (receiver side)
   ShiftTables shift;
@@ -80,8 +83,11 @@ token_kernel(const TokenArgs a) {
 
   if (a.dst != nullptr) {
     T *out = static_cast<T *>(a.dst) + t * a.lddst;
-    for (int i = lane; i < a.d; i += 32) {
-      const T *urow = U + (int64_t)i * a.ldu;
+    const T *Ux = a.U2 != nullptr ? static_cast<const T *>(a.U2) : U;
+    const int64_t ldux = a.U2 != nullptr ? a.ldu2 : a.ldu;
+    const int dx = a.U2 != nullptr ? a.d2 : a.d;
+    for (int i = lane; i < dx; i += 32) {
+      const T *urow = Ux + (int64_t)i * ldux;
       float acc = 0.f;
       for (int j = 0; j < a.k; ++j) acc = fmaf(zs[j], to_f32(urow[j]), acc);
       if (a.add_shift) {
@@ -91,6 +97,27 @@ token_kernel(const TokenArgs a) {
       out[i] = from_f32<T>(acc);
     }
   }
+}
+
+// ---- row gather: out[t, 0:kpad] = table[ids[t], 0:k] (zeros past k and for ids outside) -----
+struct GatherArgs {
+  const void *table;
+  void *out;
+  const int32_t *ids;
+  int64_t ld_table, ld_out, n, rows;
+  int32_t k, kpad;
+};
+
+template <typename T>
+__global__ void gather_rows_kernel(const GatherArgs a) {
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= a.n * a.kpad) return;
+  const int64_t t = i / a.kpad;
+  const int j = (int)(i - t * a.kpad);
+  const int64_t id = a.ids[t];
+  T v = from_f32<T>(0.f);
+  if (j < a.k && id >= 0 && id < a.rows) v = static_cast<const T *>(a.table)[id * a.ld_table + j];
+  static_cast<T *>(a.out)[t * a.ld_out + j] = v;
 }
 
 // ---- prepared tables: out [n x k] (fp32) = rows_in [n x d] U --------------------------------

@@ -86,6 +86,31 @@ bool mma_eligible(const TokenArgs &a, int32_t dtype) {
   return true;
 }
 
+ssn_status_t launch_generic_token_kernel(const TokenArgs &a, int32_t dtype, cudaStream_t stream) {
+  if (a.n == 0) return SSN_OK;
+  const int64_t blocks = (a.n + kGenericWarps - 1) / kGenericWarps;
+  if (blocks > 0x7fffffffLL) return SSN_ERR_SHAPE;
+  const size_t smem = (size_t)kGenericWarps * a.k * sizeof(float);
+  if (smem > 48 * 1024) {
+    cudaError_t e;
+    if (dtype == SSN_F32)
+      e = cudaFuncSetAttribute(token_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               (int)smem);
+    else
+      e = cudaFuncSetAttribute(token_kernel<__nv_bfloat16>,
+                               cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) {
+      cudaGetLastError();
+      return SSN_ERR_SHAPE;  // rank too large for the general kernel's shared memory
+    }
+  }
+  if (dtype == SSN_F32)
+    token_kernel<float><<<(unsigned)blocks, kGenericWarps * 32, smem, stream>>>(a);
+  else
+    token_kernel<__nv_bfloat16><<<(unsigned)blocks, kGenericWarps * 32, smem, stream>>>(a);
+  return launch_status();
+}
+
 ssn_status_t launch_token_kernel(const TokenArgs &a, int32_t dtype, cudaStream_t stream) {
   if (a.n == 0) return SSN_OK;
   if (mma_eligible(a, dtype)) {
@@ -113,27 +138,7 @@ ssn_status_t launch_token_kernel(const TokenArgs &a, int32_t dtype, cudaStream_t
       return e == cudaSuccess ? SSN_OK : SSN_ERR_CUDA;
     }
   }
-  const int64_t blocks = (a.n + kGenericWarps - 1) / kGenericWarps;
-  if (blocks > 0x7fffffffLL) return SSN_ERR_SHAPE;
-  const size_t smem = (size_t)kGenericWarps * a.k * sizeof(float);
-  if (smem > 48 * 1024) {
-    cudaError_t e;
-    if (dtype == SSN_F32)
-      e = cudaFuncSetAttribute(token_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                               (int)smem);
-    else
-      e = cudaFuncSetAttribute(token_kernel<__nv_bfloat16>,
-                               cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) {
-      cudaGetLastError();
-      return SSN_ERR_SHAPE;  // rank too large for the general kernel's shared memory
-    }
-  }
-  if (dtype == SSN_F32)
-    token_kernel<float><<<(unsigned)blocks, kGenericWarps * 32, smem, stream>>>(a);
-  else
-    token_kernel<__nv_bfloat16><<<(unsigned)blocks, kGenericWarps * 32, smem, stream>>>(a);
-  return launch_status();
+  return launch_generic_token_kernel(a, dtype, stream);
 }
 
 }  // namespace
@@ -399,6 +404,92 @@ ssn_status_t ssn_grad_project(const ssn_codec_t *codec, const void *G, int64_t l
   a.d = codec->d;
   a.k = codec->k;
   return launch_token_kernel(a, codec->dtype, static_cast<cudaStream_t>(stream));
+}
+
+ssn_status_t ssn_reparam_project(const ssn_codec_t *codec, const void *H, int64_t ldh, int64_t m,
+                                 const void *Zw, int64_t ldzw, int64_t n_tokens, void *Y,
+                                 int64_t ldy, void *coords, int64_t ldc, void *stream) {
+  ssn_status_t st = check_codec(codec);
+  if (st != SSN_OK) return st;
+  if (n_tokens < 0 || m < 1 || m > 0x7fffffffLL || ldh < m || ldzw < codec->k || ldy < codec->d) return SSN_ERR_SHAPE;
+  if (coords != nullptr && ldc < codec->k) return SSN_ERR_SHAPE;
+  if (n_tokens == 0) return SSN_OK;
+  if (H == nullptr || Zw == nullptr || Y == nullptr) return SSN_ERR_NULL;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const int sms = sm_count_of_current_device();
+  if (codec->dtype == SSN_BF16 && sms > 0 && aligned16(codec->U) && (codec->ldu & 7) == 0 && aligned16(Zw) &&
+      (ldzw & 7) == 0 && n_tokens <= 0x7fffffffLL) {
+    MmaArgs a{};
+    a.U = static_cast<const __nv_bfloat16 *>(codec->U);
+    a.ldu = codec->ldu;
+    a.d = codec->d;
+    a.k = codec->k;
+    a.B1 = static_cast<const __nv_bfloat16 *>(Zw);
+    a.ldb1 = ldzw;
+    a.d1 = (int32_t)m;
+    a.zout = static_cast<__nv_bfloat16 *>(coords);
+    a.ldzout = ldc;
+    const __nv_bfloat16 *src = static_cast<const __nv_bfloat16 *>(H);
+    __nv_bfloat16 *dst = static_cast<__nv_bfloat16 *>(Y);
+    cudaError_t e = launch_codec_umma_roundtrip_list(a, &src, &dst, &n_tokens, &ldh, &ldy, 1, sms, s, false);
+    if (e == cudaSuccess) {
+      g_launches.fetch_add(1, std::memory_order_relaxed);
+      return SSN_OK;
+    }
+    if (e != cudaErrorNotSupported) return SSN_ERR_CUDA;
+  }
+  // general path: one launch of the general kernel, the coordinates stay in fp32 in shared memory
+  TokenArgs p{};
+  p.src = H;
+  p.lds = ldh;
+  p.zout = coords;
+  p.ldzout = ldc;
+  p.dst = Y;
+  p.lddst = ldy;
+  p.U = Zw;           // contraction over the m columns of H
+  p.ldu = ldzw;
+  p.d = (int32_t)m;
+  p.U2 = codec->U;    // expansion to the d columns of Y
+  p.ldu2 = codec->ldu;
+  p.d2 = codec->d;
+  p.n = n_tokens;
+  p.k = codec->k;
+  return launch_generic_token_kernel(p, codec->dtype, s);
+}
+
+ssn_status_t ssn_head_embed(const ssn_codec_t *codec, const void *Elow, int64_t ldel,
+                            int64_t vocab_low, const int32_t *ids, const int32_t *pos,
+                            int64_t n_tokens, int32_t seq_len, void *X0, int64_t ldx,
+                            void *workspace, size_t workspace_bytes, int32_t *dev_status,
+                            void *stream) {
+  ssn_status_t st = check_codec(codec);
+  if (st != SSN_OK) return st;
+  if (n_tokens < 0 || vocab_low < 1 || ldel < codec->k || ldx < codec->d) return SSN_ERR_SHAPE;
+  if (n_tokens == 0) return SSN_OK;
+  if (Elow == nullptr || ids == nullptr || X0 == nullptr) return SSN_ERR_NULL;
+  const int32_t kpad = (codec->k + 7) / 8 * 8;
+  const size_t esz = codec->dtype == SSN_F32 ? sizeof(float) : sizeof(__nv_bfloat16);
+  if (workspace == nullptr || workspace_bytes < (size_t)n_tokens * (size_t)kpad * esz) return SSN_ERR_WORKSPACE;
+  GatherArgs g{};
+  g.table = Elow;
+  g.out = workspace;
+  g.ids = ids;
+  g.ld_table = ldel;
+  g.ld_out = kpad;
+  g.n = n_tokens;
+  g.rows = vocab_low;
+  g.k = codec->k;
+  g.kpad = kpad;
+  const int64_t total = n_tokens * kpad, blocks = (total + 255) / 256;
+  if (blocks > 0x7fffffffLL) return SSN_ERR_SHAPE;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (codec->dtype == SSN_F32)
+    gather_rows_kernel<float><<<(unsigned)blocks, 256, 0, s>>>(g);
+  else
+    gather_rows_kernel<__nv_bfloat16><<<(unsigned)blocks, 256, 0, s>>>(g);
+  st = launch_status();
+  if (st != SSN_OK) return st;
+  return ssn_decompress(codec, workspace, kpad, ids, pos, n_tokens, seq_len, X0, ldx, dev_status, stream);
 }
 
 size_t ssn_weight_reproject_workspace_bytes(const ssn_codec_t *codec, int64_t rows,

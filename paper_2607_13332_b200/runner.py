@@ -141,6 +141,28 @@ class Codec:
             return None
         return torch.empty(nbytes, dtype=torch.uint8, device=self.U.device)
 
+    def reparam_project(self, H: torch.Tensor, Zw: torch.Tensor, out: Optional[torch.Tensor] = None,
+                        coords: Optional[torch.Tensor] = None) -> torch.Tensor:
+        """Y = (H Zw) U^T for a projection stored as its factor Zw [m, k] (Eq. reparam)."""
+        n, m = H.shape
+        Y = out if out is not None else self._empty(n, self.d)
+        binding.ssn_reparam_project(self.c, H.data_ptr(), _ld(H), m, Zw.data_ptr(), _ld(Zw), n, Y.data_ptr(),
+                                    _ld(Y), coords.data_ptr() if coords is not None else 0,
+                                    _ld(coords) if coords is not None else 0, _stream())
+        return Y
+
+    def head_embed(self, Elow: torch.Tensor, ids: torch.Tensor, seq_len: int = 1,
+                   pos: Optional[torch.Tensor] = None, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+        """X0 = E[ids] + Elow[ids] U^T + P[pos]: the head stage's input with the factored embedding."""
+        n = ids.shape[0]
+        X0 = out if out is not None else self._empty(n, self.d)
+        kpad = -(-self.k // 8) * 8
+        ws = torch.empty(n * kpad * 4, dtype=torch.uint8, device=self.U.device)
+        binding.ssn_head_embed(self.c, Elow.data_ptr(), _ld(Elow), Elow.shape[0], ids.data_ptr(),
+                               pos.data_ptr() if pos is not None else 0, n, seq_len, X0.data_ptr(), _ld(X0),
+                               ws.data_ptr(), ws.numel(), self.dev_status.data_ptr(), _stream())
+        return X0
+
     def weight_reproject_list(self, weights: Sequence[torch.Tensor], side: str = "right",
                               workspace: Optional[torch.Tensor] = None) -> None:
         """In place, for weights [rows_i x d] ("right") or [d x cols_i] ("left") of any free

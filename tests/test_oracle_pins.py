@@ -354,3 +354,67 @@ def test_paper_boundary_sizes():
     assert Z.shape == (vals["tokens_8b"], 1)
     assert vals["tokens_8b"] * vals["rank_8b"] * 4 == 835_584
     assert abs(vals["d_1b"] / vals["rank_1b"] - 51.2) < 1e-12
+
+
+# ---------------------------------------------------------------------------------------
+# reparameterized forms (Eq. reparam)
+# ---------------------------------------------------------------------------------------
+def test_reparam_project_is_the_materialised_weight():
+    """Y = (H Z) U^T must be H W_p with W_p = Z U^T written out, W_p must lie in the subspace
+    (re-projecting it changes nothing), and a hand-sized case is checked with loops."""
+    rng = np.random.default_rng(11)
+    n, m, d, k = 7, 13, 24, 5
+    U = synth.subspace_basis(d, k, seed=1)
+    H, Zw = rng.standard_normal((n, m)), rng.standard_normal((m, k))
+    W = np.zeros((m, d))
+    for r in range(m):
+        for c in range(d):
+            W[r, c] = sum(Zw[r, j] * U[c, j] for j in range(k))
+    Y = oracle.reparam_project(H, Zw, U)
+    expect = np.zeros((n, d))
+    for t in range(n):
+        for c in range(d):
+            expect[t, c] = sum(H[t, r] * W[r, c] for r in range(m))
+    assert np.abs(Y - expect).max() < 1e-12
+    assert np.abs(oracle.weight_reproject(W, U, "right") - W).max() < 1e-12
+    # the coordinates the next boundary would send are H Zw: compressing Y gives them back
+    Z, _ = oracle.compress(Y, U)
+    assert np.abs(Z - H @ Zw).max() < 1e-12
+
+
+def test_reparam_factor_gradient_is_the_projected_weight_gradient():
+    """Chain rule quoted with Eq. reparam: dL/dZ = (dL/dW) U_k, checked by finite differences of
+    L = <Y, R> through reparam_project."""
+    rng = np.random.default_rng(12)
+    n, m, d, k = 5, 6, 16, 3
+    U = synth.subspace_basis(d, k, seed=2)
+    H, Zw, R = rng.standard_normal((n, m)), rng.standard_normal((m, k)), rng.standard_normal((n, d))
+    grad_W = H.T @ R                                   # dL/dW for Y = H W
+    analytic = grad_W @ U
+    eps = 1e-6
+    for r, j in ((0, 0), (3, 2), (5, 1)):
+        Zp, Zm = Zw.copy(), Zw.copy()
+        Zp[r, j] += eps
+        Zm[r, j] -= eps
+        fd = (np.sum(oracle.reparam_project(H, Zp, U) * R) - np.sum(oracle.reparam_project(H, Zm, U) * R)) / (2 * eps)
+        assert abs(fd - analytic[r, j]) < 1e-7
+
+
+def test_head_embed_is_gather_of_the_materialised_table_and_is_recovered_by_compress():
+    rng = np.random.default_rng(13)
+    V, d, k, n, S = 17, 32, 4, 40, 8
+    U = synth.subspace_basis(d, k, seed=3)
+    Elow, E, P = rng.standard_normal((V, k)), rng.standard_normal((V, d)), rng.standard_normal((S, d))
+    ids = rng.integers(0, V, n)
+    pos = oracle.token_positions(n, S)
+    X0, status = oracle.head_embed(Elow, U, E, ids, P, pos)
+    T_S = Elow @ U.T                                   # the trainable table written out
+    expect = np.stack([E[ids[t]] + T_S[ids[t]] + P[pos[t]] for t in range(n)])
+    assert status == 0 and np.abs(X0 - expect).max() < 1e-12
+    Z, _ = oracle.compress(X0, U, E, ids, P, pos)      # "entirely lossless" (Sec. 4.1)
+    assert np.abs(Z - Elow[ids]).max() < 1e-12
+    bad = ids.copy()
+    bad[2] = V
+    X1, status = oracle.head_embed(Elow, U, E, bad, P, pos)
+    assert status == oracle.STATUS_BAD_ID and np.abs(X1[2] - P[pos[2]]).max() == 0.0
+
