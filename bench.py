@@ -465,7 +465,13 @@ def run_sweep(args):
             print(json.dumps({"sweep": "reparam", "op": "reparam_project", "weight": name, "tokens": n, "m": m,
                               "d": d, "k": k, "us": round(us, 1), "GBps": round(algo / us / 1e3, 0),
                               "frac_of_measured": round(algo / us / 1e3 / peak, 3)}), flush=True)
-            del H, Zw
+            dY = (torch.randn((n, d), device="cuda", generator=gen) * 0.01).bfloat16()
+            us = timed_us(lambda: codec.reparam_grad_factor(H, dY), 5)
+            algo = n * m * 2 + n * d * 2 + m * k * 4 + d * k * 2
+            print(json.dumps({"sweep": "reparam", "op": "reparam_grad_factor", "weight": name, "tokens": n, "m": m,
+                              "d": d, "k": k, "us": round(us, 1), "GBps": round(algo / us / 1e3, 0),
+                              "frac_of_measured": round(algo / us / 1e3 / peak, 3)}), flush=True)
+            del H, Zw, dY
         E = (torch.randn((vocab, d), device="cuda", generator=gen) * 0.02).bfloat16()
         P = to_device(synth.to_storage(synth.sinusoidal_positions(seq, d), dt), dt)
         Elow = torch.randn((vocab, k), device="cuda", generator=gen).bfloat16()

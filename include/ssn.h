@@ -210,6 +210,19 @@ ssn_status_t ssn_reparam_project(const ssn_codec_t *codec, const void *H, int64_
                                  int64_t ldy, void *coords, int64_t ldc, void *stream);
 
 /*
+ * Gradient of a reparameterized projection's factor (the chain rule quoted with Eq. reparam:
+ * "the gradient for Z is (grad_W L) U_k"): with Y = (H Zw) U^T and dY = dL/dY,
+ *     dZw [m x k] = H^T (dY U)        (fp32 output, written, not accumulated)
+ *   workspace  device scratch of n * kpad * sizeof(element) bytes, kpad = k rounded up to 8,
+ *              16-byte aligned: the coordinates dY U (in the storage dtype).
+ * E and P of the codec are not used.
+ */
+ssn_status_t ssn_reparam_grad_factor(const ssn_codec_t *codec, const void *H, int64_t ldh,
+                                     int64_t m, const void *dY, int64_t lddy, int64_t n_tokens,
+                                     float *dZw, int64_t lddz, void *workspace,
+                                     size_t workspace_bytes, void *stream);
+
+/*
  * Head-stage input of the reparameterized SSN (Sec. 4.1: the trainable embedding is factored as
  * T_S = Elow U_k^T "with every projection and the embedding parameterized through U_k"):
  *     X0[t,:] = E[ids[t],:] + Elow[ids[t],:] U^T + P[pos(t),:]

@@ -117,6 +117,12 @@ def reparam_project(H: np.ndarray, Zw: np.ndarray, U: np.ndarray) -> np.ndarray:
     return (H @ np.asarray(Zw, dtype=np.float64)) @ np.asarray(U, dtype=np.float64).T
 
 
+def reparam_grad_factor(H: np.ndarray, dY: np.ndarray, U: np.ndarray) -> np.ndarray:
+    """The chain rule quoted with Eq. reparam: dL/dZw = (dL/dW) U_k with dL/dW = H^T dY for Y = H W."""
+    H = np.asarray(H, dtype=np.float64)
+    return H.T @ (np.asarray(dY, dtype=np.float64) @ np.asarray(U, dtype=np.float64))
+
+
 def head_embed(Elow: np.ndarray, U: np.ndarray, E=None, ids=None, P=None, pos=None):
     """Head-stage input with the factored trainable embedding T_S = Elow U_k^T (Sec. 4.1):
     X0[t] = T_fixed[ids[t]] + Elow[ids[t]] U_k^T + PE[pos[t]].  A token whose id is outside Elow

@@ -68,6 +68,7 @@ _SIGNATURES = {
     "ssn_weight_reproject_left_static": (_i32, [_codec_p, _vp, _i64, _i64, _vp]),
     "ssn_prepare_tables": (_i32, [_codec_p, _vp, _i64, _vp, _i64, _vp]),
     "ssn_reparam_project": (_i32, [_codec_p, _vp, _i64, _i64, _vp, _i64, _i64, _vp, _i64, _vp, _i64, _vp]),
+    "ssn_reparam_grad_factor": (_i32, [_codec_p, _vp, _i64, _i64, _vp, _i64, _i64, _vp, _i64, _vp, _sz, _vp]),
     "ssn_head_embed": (_i32, [_codec_p, _vp, _i64, _i64, _vp, _vp, _i64, _i32, _vp, _i64, _vp, _sz, _vp, _vp]),
     "ssn_weight_reproject_list": (_i32, [_codec_p, ctypes.POINTER(_vp), ctypes.POINTER(_i64),
                                          ctypes.POINTER(_i64), _i32, _i32, _vp, _sz, _vp]),
@@ -182,6 +183,14 @@ def ssn_reparam_project(codec: ssn_codec_t, H: int, ldh: int, m: int, Zw: int, l
     _check(_lib.ssn_reparam_project(ctypes.byref(codec), H or None, ldh, m, Zw or None, ldzw, n_tokens,
                                     Y or None, ldy, coords or None, ldc, stream or None),
            "ssn_reparam_project")
+
+
+def ssn_reparam_grad_factor(codec: ssn_codec_t, H: int, ldh: int, m: int, dY: int, lddy: int, n_tokens: int,
+                            dZw: int, lddz: int, workspace: int, workspace_bytes: int, stream: int = 0) -> None:
+    """dZw [m x k] (fp32) = H^T (dY U): the gradient of a reparameterized projection's factor."""
+    _check(_lib.ssn_reparam_grad_factor(ctypes.byref(codec), H or None, ldh, m, dY or None, lddy, n_tokens,
+                                        dZw or None, lddz, workspace or None, workspace_bytes, stream or None),
+           "ssn_reparam_grad_factor")
 
 
 def ssn_head_embed(codec: ssn_codec_t, Elow: int, ldel: int, vocab_low: int, ids: int, pos: int,

@@ -5,6 +5,7 @@
 #include "codec_umma.cuh"
 #include "codec_umma_roundtrip.cuh"
 #include "codec_umma_expand.cuh"
+#include "codec_umma_tokens.cuh"
 
 
 #include "codec_mma_launch.h"
@@ -414,6 +415,57 @@ cudaError_t launch_codec_umma_expand(const MmaArgs &a, bool shift, int sm_count,
   if (has_e) return launch_umma_expand_one<1, true, false>(a, geo, maps, sm_count, stream);
   if (has_p) return launch_umma_expand_one<1, false, true>(a, geo, maps, sm_count, stream);
   return launch_umma_expand_one<1, false, false>(a, geo, maps, sm_count, stream);
+}
+
+namespace {
+template <int NTP>
+cudaError_t launch_tokens_ntp(const TokensArgs &t, const UmmaTokensMaps &maps, int grid, cudaStream_t stream) {
+  auto kernel = codec_umma_tokens_kernel<NTP>;
+  constexpr int smem = UmmaTokensConfig<NTP>::kSmemBytes;
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  kernel<<<(unsigned)grid, kTokensThreads, smem, stream>>>(t, maps);
+  return cudaGetLastError();
+}
+}  // namespace
+
+cudaError_t launch_codec_umma_tokens(const __nv_bfloat16 *H, int64_t ldh, const __nv_bfloat16 *C, int64_t ldc,
+                                     float *out, int64_t ldout, int64_t n, int32_t m, int32_t k,
+                                     int sm_count, cudaStream_t stream) {
+  if (H == nullptr || C == nullptr || out == nullptr || k > 128 || k < 1 || m < 1) return cudaErrorNotSupported;
+  if (n < 4 * kUmmaTile || n > 0x7fffffffLL) return cudaErrorNotSupported;
+  UmmaTokensMaps maps;
+  if (!make_sw128_map(&maps.h, H, n, m, ldh, kUmmaCols)) return cudaErrorNotSupported;
+  if (!make_sw128_map(&maps.c, C, n, k, ldc, kUmmaCols)) return cudaErrorNotSupported;
+  if (!make_sw128_map(&maps.c_wide, C, n, k <= 64 ? 64 : 128, ldc, kUmmaCols)) return cudaErrorNotSupported;
+  const int nblk = (m + kUmmaTile - 1) / kUmmaTile;
+  const int64_t nstage = (n + kUmmaCols - 1) / kUmmaCols;
+  int64_t splits = sm_count / nblk;
+  if (splits < 1) splits = 1;
+  if (splits > nstage) splits = nstage;
+  TokensArgs t{};
+  t.out = out;
+  t.ldout = ldout;
+  t.n = n;
+  t.m = m;
+  t.k = k;
+  t.splits = (int32_t)splits;
+  if (splits > 1) {
+    cudaError_t e = cudaMemset2DAsync(out, (size_t)ldout * sizeof(float), 0, (size_t)k * sizeof(float), (size_t)m, stream);
+    if (e != cudaSuccess) return e;
+  }
+  const int grid = (int)(nblk * splits);
+  const int ntp = 2 * ((k + 15) / 16);
+  if (ntp <= 2) return launch_tokens_ntp<2>(t, maps, grid, stream);
+  if (ntp <= 4) return launch_tokens_ntp<4>(t, maps, grid, stream);
+  if (ntp <= 6) return launch_tokens_ntp<6>(t, maps, grid, stream);
+  if (ntp <= 8) return launch_tokens_ntp<8>(t, maps, grid, stream);
+  if (ntp <= 12) return launch_tokens_ntp<12>(t, maps, grid, stream);
+  return launch_tokens_ntp<16>(t, maps, grid, stream);
 }
 
 bool codec_mma_supports(int d, int k) {

@@ -42,6 +42,13 @@ cudaError_t launch_codec_umma_roundtrip_list(const MmaArgs &a, const __nv_bfloat
                                              const int64_t *lds, const int64_t *lddst, int count,
                                              int sm_count, cudaStream_t stream, bool left);
 
+// out [m x k] (fp32) = H^T C on tcgen05 (H: [n x m], C: [n x k], both bf16); cudaErrorNotSupported
+// when the shapes or alignments are not the kernel's, and nothing has been launched then.  The
+// output is zeroed on the stream first when several CTAs share a row block.
+cudaError_t launch_codec_umma_tokens(const __nv_bfloat16 *H, int64_t ldh, const __nv_bfloat16 *C, int64_t ldc,
+                                     float *out, int64_t ldout, int64_t n, int32_t m, int32_t k,
+                                     int sm_count, cudaStream_t stream);
+
 // mode: 1 = project, 2 = expand, 3 = project then expand (shift must be false).
 cudaError_t launch_codec_mma(const MmaArgs &a, bool shift, int mode, int sm_count,
                              cudaStream_t stream);

@@ -120,6 +120,25 @@ __global__ void gather_rows_kernel(const GatherArgs a) {
   static_cast<T *>(a.out)[t * a.ld_out + j] = v;
 }
 
+// ---- contraction over tokens: out [m x k] (fp32) = H^T C, H [n x m], C [n x k] ---------------
+struct TokensContractArgs {
+  const void *H, *C;
+  float *out;
+  int64_t ldh, ldc, ldout, n;
+  int32_t m, k;
+};
+
+// One thread per output element, 32 rows x 8 columns per block; the loads of H are coalesced.
+template <typename T>
+__global__ void __launch_bounds__(256) tokens_contract_kernel(const TokensContractArgs a) {
+  const int r = blockIdx.x * 32 + (threadIdx.x & 31), j = blockIdx.y * 8 + (threadIdx.x >> 5);
+  if (r >= a.m || j >= a.k) return;
+  const T *H = static_cast<const T *>(a.H), *C = static_cast<const T *>(a.C);
+  float acc = 0.f;
+  for (int64_t t = 0; t < a.n; ++t) acc = fmaf(to_f32(H[t * a.ldh + r]), to_f32(C[t * a.ldc + j]), acc);
+  a.out[(int64_t)r * a.ldout + j] = acc;
+}
+
 // ---- prepared tables: out [n x k] (fp32) = rows_in [n x d] U --------------------------------
 struct TableArgs {
   const void *rows_in;   // E or P

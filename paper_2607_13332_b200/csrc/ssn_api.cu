@@ -457,6 +457,59 @@ ssn_status_t ssn_reparam_project(const ssn_codec_t *codec, const void *H, int64_
   return launch_generic_token_kernel(p, codec->dtype, s);
 }
 
+ssn_status_t ssn_reparam_grad_factor(const ssn_codec_t *codec, const void *H, int64_t ldh, int64_t m,
+                                     const void *dY, int64_t lddy, int64_t n_tokens, float *dZw,
+                                     int64_t lddz, void *workspace, size_t workspace_bytes,
+                                     void *stream) {
+  ssn_status_t st = check_codec(codec);
+  if (st != SSN_OK) return st;
+  if (n_tokens < 1 || m < 1 || m > 0x7fffffffLL || ldh < m || lddy < codec->d || lddz < codec->k) return SSN_ERR_SHAPE;
+  if (H == nullptr || dY == nullptr || dZw == nullptr) return SSN_ERR_NULL;
+  const int32_t kpad = (codec->k + 7) / 8 * 8;
+  const size_t esz = codec->dtype == SSN_F32 ? sizeof(float) : sizeof(__nv_bfloat16);
+  if (workspace == nullptr || workspace_bytes < (size_t)n_tokens * (size_t)kpad * esz) return SSN_ERR_WORKSPACE;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  TokenArgs p{};      // C = dY U: "the backward pass uses the same compression"
+  p.src = dY;
+  p.lds = lddy;
+  p.zout = workspace;
+  p.ldzout = kpad;
+  p.U = codec->U;
+  p.ldu = codec->ldu;
+  p.n = n_tokens;
+  p.d = codec->d;
+  p.k = codec->k;
+  st = launch_token_kernel(p, codec->dtype, s);
+  if (st != SSN_OK) return st;
+  const int sms = sm_count_of_current_device();
+  if (codec->dtype == SSN_BF16 && sms > 0) {
+    cudaError_t e = launch_codec_umma_tokens(static_cast<const __nv_bfloat16 *>(H), ldh,
+                                             static_cast<const __nv_bfloat16 *>(workspace), kpad, dZw, lddz,
+                                             n_tokens, (int32_t)m, codec->k, sms, s);
+    if (e == cudaSuccess) {
+      g_launches.fetch_add(1, std::memory_order_relaxed);
+      return SSN_OK;
+    }
+    if (e != cudaErrorNotSupported) return SSN_ERR_CUDA;
+  }
+  TokensContractArgs c{};
+  c.H = H;
+  c.C = workspace;
+  c.out = dZw;
+  c.ldh = ldh;
+  c.ldc = kpad;
+  c.ldout = lddz;
+  c.n = n_tokens;
+  c.m = (int32_t)m;
+  c.k = codec->k;
+  dim3 grid((unsigned)((m + 31) / 32), (unsigned)((codec->k + 7) / 8));
+  if (codec->dtype == SSN_F32)
+    tokens_contract_kernel<float><<<grid, 256, 0, s>>>(c);
+  else
+    tokens_contract_kernel<__nv_bfloat16><<<grid, 256, 0, s>>>(c);
+  return launch_status();
+}
+
 ssn_status_t ssn_head_embed(const ssn_codec_t *codec, const void *Elow, int64_t ldel,
                             int64_t vocab_low, const int32_t *ids, const int32_t *pos,
                             int64_t n_tokens, int32_t seq_len, void *X0, int64_t ldx,

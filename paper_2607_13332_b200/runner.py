@@ -151,6 +151,16 @@ class Codec:
                                     _ld(coords) if coords is not None else 0, _stream())
         return Y
 
+    def reparam_grad_factor(self, H: torch.Tensor, dY: torch.Tensor) -> torch.Tensor:
+        """dZw [m, k] (fp32) = H^T (dY U) for a projection stored as its factor (Eq. reparam)."""
+        n, m = H.shape
+        out = torch.empty((m, self.k), dtype=torch.float32, device=self.U.device)
+        kpad = -(-self.k // 8) * 8
+        ws = torch.empty(n * kpad * 4, dtype=torch.uint8, device=self.U.device)
+        binding.ssn_reparam_grad_factor(self.c, H.data_ptr(), _ld(H), m, dY.data_ptr(), _ld(dY), n,
+                                        out.data_ptr(), self.k, ws.data_ptr(), ws.numel(), _stream())
+        return out
+
     def head_embed(self, Elow: torch.Tensor, ids: torch.Tensor, seq_len: int = 1,
                    pos: Optional[torch.Tensor] = None, out: Optional[torch.Tensor] = None) -> torch.Tensor:
         """X0 = E[ids] + Elow[ids] U^T + P[pos]: the head stage's input with the factored embedding."""

@@ -74,6 +74,25 @@ def test_head_embed(batch, seq_len, d, k, vocab, dt):
     assert_close(host64(Z, dt)[good], f64(Elow0, dt)[ids_np[good]], dt, "compress(head embed)", tol=2e-2 if dt == synth.BF16 else 1e-4)
 
 
+@pytest.mark.parametrize("n,m,d,k,dt", CASES + [(65536, 4096, 4096, 40, synth.BF16), (1100, 200, 256, 24, synth.BF16)])
+def test_reparam_grad_factor(n, m, d, k, dt):
+    """dZw = H^T (dY U): tensor-core shapes (several CTAs per row block add their partial sums)
+    and general ones, against the oracle."""
+    if n * m > 1 << 28:
+        pytest.skip("too large for the oracle in a unit test")
+    rng = np.random.default_rng(n + m + 3 * d + k)
+    U0 = synth.to_storage(synth.subspace_basis(d, k, seed=m + k), dt)
+    H0 = synth.to_storage(rng.standard_normal((n, m)) * 0.5, dt)
+    dY0 = synth.to_storage(rng.standard_normal((n, d)) * 0.01, dt)
+    codec = Codec(dt, to_device(U0, dt))
+    got = codec.reparam_grad_factor(to_device(H0, dt), to_device(dY0, dt))
+    expect = oracle.reparam_grad_factor(f64(H0, dt), f64(dY0, dt), f64(U0, dt))
+    assert_close(got.double().cpu().numpy(), expect, dt, "dZw = H^T (dY U)")
+    # a second call overwrites, it does not accumulate
+    got2 = codec.reparam_grad_factor(to_device(H0, dt), to_device(dY0, dt))
+    assert_close(got2.double().cpu().numpy(), expect, dt, "second call")
+
+
 def test_reparam_argument_errors():
     dt, d, k = synth.BF16, 256, 8
     codec = Codec(dt, to_device(synth.to_storage(synth.subspace_basis(d, k, seed=3), dt), dt))
@@ -88,4 +107,11 @@ def test_reparam_argument_errors():
     assert ok(H.data_ptr(), 64, 64, Zw.data_ptr(), k, 16, Y.data_ptr(), d - 1, None, 0, None) == binding.SSN_ERR_SHAPE
     assert ok(None, 64, 64, Zw.data_ptr(), k, 16, Y.data_ptr(), d, None, 0, None) == binding.SSN_ERR_NULL
     assert ok(H.data_ptr(), 64, 64, Zw.data_ptr(), k, 0, Y.data_ptr(), d, None, 0, None) == binding.SSN_OK
+    g = binding.raw("ssn_reparam_grad_factor")
+    dZ = torch.zeros((64, k), dtype=torch.float32, device="cuda")
+    ws = torch.zeros(16 * 8 * 2, dtype=torch.uint8, device="cuda")
+    assert g(codec.c, H.data_ptr(), 64, 64, Y.data_ptr(), d, 16, dZ.data_ptr(), k, ws.data_ptr(), ws.numel(), None) == binding.SSN_OK
+    assert g(codec.c, H.data_ptr(), 64, 64, Y.data_ptr(), d, 16, dZ.data_ptr(), k, None, 0, None) == binding.SSN_ERR_WORKSPACE
+    assert g(codec.c, H.data_ptr(), 64, 64, Y.data_ptr(), d, 16, dZ.data_ptr(), k - 1, ws.data_ptr(), ws.numel(), None) == binding.SSN_ERR_SHAPE
+    assert g(codec.c, H.data_ptr(), 64, 64, None, d, 16, dZ.data_ptr(), k, ws.data_ptr(), ws.numel(), None) == binding.SSN_ERR_NULL
     torch.cuda.synchronize()

@@ -391,6 +391,7 @@ def test_reparam_factor_gradient_is_the_projected_weight_gradient():
     H, Zw, R = rng.standard_normal((n, m)), rng.standard_normal((m, k)), rng.standard_normal((n, d))
     grad_W = H.T @ R                                   # dL/dW for Y = H W
     analytic = grad_W @ U
+    assert np.abs(oracle.reparam_grad_factor(H, R, U) - analytic).max() < 1e-12
     eps = 1e-6
     for r, j in ((0, 0), (3, 2), (5, 1)):
         Zp, Zm = Zw.copy(), Zw.copy()
