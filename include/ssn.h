@@ -204,6 +204,8 @@ ssn_status_t ssn_weight_reproject_list(const ssn_codec_t *codec, void *const *W_
  *   coords     optional [n x k] output of the coordinates H Zw (storage dtype, ldc >= k), or NULL
  * The coordinates stay in fp32 between the two products on every path.
  * H and Y must not overlap.  E and P of the codec are not used.
+ * The activation gradient of the same layer, dH [n x m] = (dY U) Zw^T, is this call with the two
+ * factors exchanged: a codec whose U is Zw (d = m) and Zw := U ([d x k], m := d), H := dY.
  */
 ssn_status_t ssn_reparam_project(const ssn_codec_t *codec, const void *H, int64_t ldh, int64_t m,
                                  const void *Zw, int64_t ldzw, int64_t n_tokens, void *Y,

@@ -93,6 +93,19 @@ def test_reparam_grad_factor(n, m, d, k, dt):
     assert_close(got2.double().cpu().numpy(), expect, dt, "second call")
 
 
+def test_activation_gradient_is_the_same_call_with_the_factors_exchanged():
+    """dH = (dY U) Zw^T: ssn_reparam_project on a codec whose basis is Zw, with U as the factor."""
+    dt, n, m, d, k = synth.BF16, 1536, 1024, 512, 40
+    rng = np.random.default_rng(7)
+    U0 = synth.to_storage(synth.subspace_basis(d, k, seed=9), dt)
+    Zw0 = synth.to_storage(rng.standard_normal((m, k)) / np.sqrt(m), dt)
+    dY0 = synth.to_storage(rng.standard_normal((n, d)) * 0.01, dt)
+    swapped = Codec(dt, to_device(Zw0, dt))              # "U" of this codec is Zw: [m x k]
+    dH = swapped.reparam_project(to_device(dY0, dt), to_device(U0, dt))
+    expect = (f64(dY0, dt) @ f64(U0, dt)) @ f64(Zw0, dt).T
+    assert_close(host64(dH, dt), expect, dt, "dH = (dY U) Zw^T")
+
+
 def test_reparam_argument_errors():
     dt, d, k = synth.BF16, 256, 8
     codec = Codec(dt, to_device(synth.to_storage(synth.subspace_basis(d, k, seed=3), dt), dt))
