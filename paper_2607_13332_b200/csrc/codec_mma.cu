@@ -444,9 +444,17 @@ cudaError_t launch_codec_umma_tokens(const __nv_bfloat16 *H, int64_t ldh, const 
   if (!make_sw128_map(&maps.c_wide, C, n, k <= 64 ? 64 : 128, ldc, kUmmaCols)) return cudaErrorNotSupported;
   const int nblk = (m + kUmmaTile - 1) / kUmmaTile;
   const int64_t nstage = (n + kUmmaCols - 1) / kUmmaCols;
-  int64_t splits = sm_count / nblk;
-  if (splits < 1) splits = 1;
-  if (splits > nstage) splits = nstage;
+  // CTAs per column block: the count (up to 16) that fills whole waves of SMs best
+  int64_t splits = 1;
+  double best = 0.0;
+  for (int64_t s = 1; s <= 16 && s <= nstage; ++s) {
+    const int64_t ctas = nblk * s, waves = (ctas + sm_count - 1) / sm_count;
+    const double fill = (double)ctas / (double)(waves * sm_count);
+    if (fill > best + 1e-9) {
+      best = fill;
+      splits = s;
+    }
+  }
   TokensArgs t{};
   t.out = out;
   t.ldout = ldout;
