@@ -32,6 +32,9 @@ SHAPES = [
     (16, 128, 1024, 96, 500),    # 64 < k <= 128 on the expansion kernel, 8 x 16 tiles
     (8, 256, 512, 128, 300),
     (24, 64, 256, 72, 100),
+    (8, 128, 64, 8, 40),         # d = 64: a single stage per tile, pairs cannot split it
+    (9, 128, 128, 1, 40),        # k = 1, odd number of tiles
+    (8, 128, 128, 16, 40),
 ]
 
 
