@@ -61,7 +61,7 @@ def parse_args():
                          "the E and P rows (the default step gathers; the table variant is always "
                          "timed beside it as compress_prepared_tables)")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
-    ap.add_argument("--sweep", choices=["compress", "reproject", "reparam"], default=None,
+    ap.add_argument("--sweep", choices=["compress", "reproject", "reparam", "wire"], default=None,
                     help="instead of the step: time the compress sweep (d, k, tokens) or the "
                          "re-projection sweep (k, weight shape, 32 layers); one JSON line per point")
     return ap.parse_args()
@@ -403,7 +403,7 @@ def run_sweep(args):
 
     import __graft_entry__ as entry
     entry.build()
-    from paper_2607_13332_b200 import synth
+    from paper_2607_13332_b200 import binding, synth
     from paper_2607_13332_b200.runner import Codec, to_device
 
     peak, _ = measured_hbm_peak()
@@ -485,6 +485,48 @@ def run_sweep(args):
         print(json.dumps({"sweep": "reparam", "op": "head_embed", "tokens": n, "d": d, "k": k,
                           "us": round(us, 1), "GBps": round(algo / us / 1e3, 0),
                           "frac_of_measured": round(algo / us / 1e3 / peak, 3)}), flush=True)
+    elif args.sweep == "wire":
+        # wire rows (k fp32 coordinates + the token id) at the benchmark's stage boundary, next to the
+        # storage-dtype calls of the step; ranks 24 and 40: decompress with one / two coordinate groups
+        d, n = 4096, 65536
+        wl = synth.STAGE_8B
+        ids_np = synth.token_ids(wl, 3)
+        ids = torch.from_numpy(ids_np).cuda()
+        uniq = int(np.unique(ids_np).size)
+        E = (torch.randn((vocab, d), device="cuda", generator=gen) * 0.02).bfloat16()
+        P = to_device(synth.to_storage(synth.sinusoidal_positions(seq, d), dt), dt)
+        X = torch.randn((n, d), device="cuda", generator=gen).bfloat16()
+        Xh = torch.empty_like(X)
+        for k in (24, 40):
+            U = to_device(synth.to_storage(synth.subspace_basis(d, k, 1), dt), dt)
+            codec, codec_t = Codec(dt, U, E, P), Codec(dt, U, E, P)
+            codec_t.prepare_tables()
+            wire = codec.wire_buffer(n, True)
+            dZ = torch.empty((n, k), dtype=torch.float32, device="cuda")
+            Z = torch.empty((n, k), dtype=torch.bfloat16, device="cuda")
+            nbytes = binding.ssn_decompress_wire_workspace_bytes(codec.c, n, True)
+            ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+            rows_in = n * d * 2 + uniq * d * 2 + seq * d * 2 + d * k * 2 + n * 4
+            points = (
+                ("compress_wire", lambda: codec.compress_wire(X, ids, seq_len=seq, with_ids=True, out=wire),
+                 rows_in + n * (k + 1) * 4),
+                ("compress_wire, prepared tables",
+                 lambda: codec_t.compress_wire(X, ids, seq_len=seq, with_ids=True, out=wire),
+                 n * d * 2 + n * 4 + (uniq + seq) * k * 4 + d * k * 2 + n * (k + 1) * 4),
+                ("compress (bf16 rows)", lambda: codec.compress(X, ids, seq_len=seq, out=Z), rows_in + n * k * 2),
+                ("grad_project_wire", lambda: codec.grad_project_wire(X, out=dZ), n * d * 2 + d * k * 2 + n * k * 4),
+                ("decompress_wire",
+                 lambda: codec.decompress_wire(wire, seq_len=seq, with_ids=True, out=Xh, workspace=ws),
+                 n * (k + 1) * 4 + uniq * d * 2 + seq * d * 2 + d * k * 2 + n * d * 2),
+                ("decompress (bf16 rows)", lambda: codec.decompress(Z, ids, seq_len=seq, out=Xh),
+                 n * k * 2 + n * 4 + uniq * d * 2 + seq * d * 2 + d * k * 2 + n * d * 2),
+            )
+            for name, fn, algo in points:
+                us = timed_us(fn, 10)
+                print(json.dumps({"sweep": "wire", "op": name, "tokens": n, "d": d, "k": k, "us": round(us, 1),
+                                  "GBps": round(algo / us / 1e3, 0),
+                                  "frac_of_measured": round(algo / us / 1e3 / peak, 3),
+                                  "status": codec.take_status() | codec_t.take_status()}), flush=True)
     else:
         d = 4096
         for k in synth.REPROJECT_RANKS:

@@ -242,6 +242,45 @@ ssn_status_t ssn_head_embed(const ssn_codec_t *codec, const void *Elow, int64_t 
                             void *stream);
 
 /*
+ * Wire rows.  The paper's bandwidth estimate (Sec. 3.5, "Stability Under Bandwidth
+ * Constraints", the paragraph on the estimated communication) counts the boundary tensors in FP32, and the receiver of a forward activation needs the token ids for
+ * T_fixed[ids]; these three calls produce and consume that form directly, whatever the storage
+ * dtype of X:
+ *     row t of `wire` = k fp32 coordinates, then (with_ids != 0) the token id as one int32 word
+ * `wire` is a device buffer of 32-bit words with leading dimension ldw >= k + (with_ids ? 1 : 0)
+ * words (any larger pitch leaves room for the caller's own header words; rows 16-byte aligned
+ * with ldw % 4 == 0 get vector stores).  The coordinates are the fp32 accumulator values: for a
+ * bf16 codec they are NOT rounded to bf16 on the way.
+ *
+ * ssn_compress_wire       as ssn_compress (prepared tables included); with_ids needs ids.
+ * ssn_grad_project_wire   dZ = G U as fp32 rows (no ids).
+ * ssn_decompress_wire     as ssn_decompress from wire rows; with_ids != 0: the ids are taken from
+ *                         the rows and the `ids` argument is ignored.  A bf16 codec with
+ *                         2 * kpad <= 128 (kpad = k rounded up to 8) runs on the tensor cores
+ *                         with the fp32 coordinates split into a bf16 head and a bf16 remainder
+ *                         (rank 2 * kpad against the basis repeated twice), so no precision of
+ *                         the coordinates is dropped before the single rounding of X^; for that
+ *                         the call needs a 256-byte aligned workspace of
+ *                         ssn_decompress_wire_workspace_bytes() bytes.  With a smaller (or
+ *                         misaligned) workspace the general kernel runs; with_ids always needs
+ *                         at least n_tokens * 4 bytes (rounded up to 256).
+ * Errors as for the calls they mirror, plus SSN_ERR_WORKSPACE.
+ */
+ssn_status_t ssn_compress_wire(const ssn_codec_t *codec, const void *X, int64_t ldx,
+                               const int32_t *ids, const int32_t *pos, int64_t n_tokens,
+                               int32_t seq_len, void *wire, int64_t ldw, int32_t with_ids,
+                               int32_t *dev_status, void *stream);
+ssn_status_t ssn_grad_project_wire(const ssn_codec_t *codec, const void *G, int64_t ldg,
+                                   int64_t n_tokens, float *dZ, int64_t ldw, void *stream);
+size_t ssn_decompress_wire_workspace_bytes(const ssn_codec_t *codec, int64_t n_tokens,
+                                           int32_t with_ids);
+ssn_status_t ssn_decompress_wire(const ssn_codec_t *codec, const void *wire, int64_t ldw,
+                                 int32_t with_ids, const int32_t *ids, const int32_t *pos,
+                                 int64_t n_tokens, int32_t seq_len, void *Xhat, int64_t ldx,
+                                 void *workspace, size_t workspace_bytes, int32_t *dev_status,
+                                 void *stream);
+
+/*
  * LEFT re-projection of ONE weight, W [d x cols] <- U (U^T W), without a caller workspace.
  * (The paper has no counterpart: this is a packaging variant of ssn_weight_reproject.)
  *

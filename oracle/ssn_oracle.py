@@ -25,7 +25,8 @@ gather, isometry at k = d, exact round trip inside the subspace, adjoint and fin
 identities, projector identities, explicit d x d projector, element-by-element loops on tiny
 shapes; for the reparameterized forms (Eq. reparam): the materialised weight W_p = Z U^T, its
 membership of the subspace, loops, and the exact recovery of the factored embedding's coordinates
-by compress.  No function here is left unpinned.
+by compress; for the wire rows: IEEE-754 bit patterns typed by hand, the id word, the round trip
+within half an fp32 ulp.  No function here is left unpinned.
 """
 
 from __future__ import annotations
@@ -134,3 +135,20 @@ def head_embed(Elow: np.ndarray, U: np.ndarray, E=None, ids=None, P=None, pos=No
     Z[ok] = Elow[ids[ok]]
     return decompress(Z, U, E, ids, P, pos)
 
+
+
+def wire_rows(Z: np.ndarray, ids=None) -> np.ndarray:
+    """Wire form of the boundary tensor (Sec. 3.5 sizes the boundary traffic in FP32): row t holds
+    the k coordinates rounded to the nearest float32, as 32-bit words, followed (when ids is given)
+    by the token id as an int32 word.  Returns an int32 array [n, k] or [n, k + 1]."""
+    words = np.asarray(Z, dtype=np.float64).astype(np.float32).view(np.int32)
+    if ids is None:
+        return words.copy()
+    return np.concatenate([words, np.asarray(ids, dtype=np.int32).reshape(-1, 1)], axis=1)
+
+
+def wire_unpack(wire: np.ndarray, k: int, with_ids: bool):
+    """Inverse of wire_rows: (coordinates as float64 [n, k], ids as int64 [n] or None)."""
+    wire = np.ascontiguousarray(np.asarray(wire, dtype=np.int32))
+    Z = wire[:, :k].copy().view(np.float32).astype(np.float64)
+    return Z, (wire[:, k].astype(np.int64) if with_ids else None)

@@ -70,6 +70,11 @@ _SIGNATURES = {
     "ssn_reparam_project": (_i32, [_codec_p, _vp, _i64, _i64, _vp, _i64, _i64, _vp, _i64, _vp, _i64, _vp]),
     "ssn_reparam_grad_factor": (_i32, [_codec_p, _vp, _i64, _i64, _vp, _i64, _i64, _vp, _i64, _vp, _sz, _vp]),
     "ssn_head_embed": (_i32, [_codec_p, _vp, _i64, _i64, _vp, _vp, _i64, _i32, _vp, _i64, _vp, _sz, _vp, _vp]),
+    "ssn_compress_wire": (_i32, [_codec_p, _vp, _i64, _vp, _vp, _i64, _i32, _vp, _i64, _i32, _vp, _vp]),
+    "ssn_grad_project_wire": (_i32, [_codec_p, _vp, _i64, _i64, _vp, _i64, _vp]),
+    "ssn_decompress_wire_workspace_bytes": (_sz, [_codec_p, _i64, _i32]),
+    "ssn_decompress_wire": (_i32, [_codec_p, _vp, _i64, _i32, _vp, _vp, _i64, _i32, _vp, _i64, _vp, _sz,
+                                   _vp, _vp]),
     "ssn_weight_reproject_list": (_i32, [_codec_p, ctypes.POINTER(_vp), ctypes.POINTER(_i64),
                                          ctypes.POINTER(_i64), _i32, _i32, _vp, _sz, _vp]),
     "ssn_static_scratch_bytes": (_sz, []),
@@ -200,6 +205,34 @@ def ssn_head_embed(codec: ssn_codec_t, Elow: int, ldel: int, vocab_low: int, ids
     _check(_lib.ssn_head_embed(ctypes.byref(codec), Elow or None, ldel, vocab_low, ids or None, pos or None,
                                n_tokens, seq_len, X0 or None, ldx, workspace or None, workspace_bytes,
                                dev_status or None, stream or None), "ssn_head_embed")
+
+
+def ssn_compress_wire(codec: ssn_codec_t, X: int, ldx: int, ids: int, pos: int, n_tokens: int, seq_len: int,
+                      wire: int, ldw: int, with_ids: bool, dev_status: int = 0, stream: int = 0) -> None:
+    """ssn_compress into wire rows: k fp32 coordinates, then (with_ids) the token id as int32."""
+    _check(_lib.ssn_compress_wire(ctypes.byref(codec), X or None, ldx, ids or None, pos or None, n_tokens,
+                                  seq_len, wire or None, ldw, 1 if with_ids else 0, dev_status or None,
+                                  stream or None), "ssn_compress_wire")
+
+
+def ssn_grad_project_wire(codec: ssn_codec_t, G: int, ldg: int, n_tokens: int, dZ: int, ldw: int,
+                          stream: int = 0) -> None:
+    """dZ = G U as fp32 wire rows."""
+    _check(_lib.ssn_grad_project_wire(ctypes.byref(codec), G or None, ldg, n_tokens, dZ or None, ldw,
+                                      stream or None), "ssn_grad_project_wire")
+
+
+def ssn_decompress_wire_workspace_bytes(codec: ssn_codec_t, n_tokens: int, with_ids: bool) -> int:
+    return int(_lib.ssn_decompress_wire_workspace_bytes(ctypes.byref(codec), n_tokens, 1 if with_ids else 0))
+
+
+def ssn_decompress_wire(codec: ssn_codec_t, wire: int, ldw: int, with_ids: bool, ids: int, pos: int,
+                        n_tokens: int, seq_len: int, Xhat: int, ldx: int, workspace: int, workspace_bytes: int,
+                        dev_status: int = 0, stream: int = 0) -> None:
+    """ssn_decompress from wire rows (the ids come from the rows when with_ids)."""
+    _check(_lib.ssn_decompress_wire(ctypes.byref(codec), wire or None, ldw, 1 if with_ids else 0, ids or None,
+                                    pos or None, n_tokens, seq_len, Xhat or None, ldx, workspace or None,
+                                    workspace_bytes, dev_status or None, stream or None), "ssn_decompress_wire")
 
 
 def ssn_prepare_tables(codec: ssn_codec_t, EU: int, ldeu: int, PU: int, ldpu: int,

@@ -243,7 +243,8 @@ cudaError_t launch_umma_ntp(const MmaArgs &a, bool has_e, bool has_p, const Umma
 // kernel instead: small batches, k > 128, d not a multiple of 64, explicit or
 // wrapping positions inside a 128-token tile, no tensor map.
 cudaError_t launch_codec_umma_project(const MmaArgs &a, bool shift, int sm_count, cudaStream_t stream) {
-  if (a.zout == nullptr || a.dst != nullptr || a.src == nullptr) return cudaErrorNotSupported;
+  if ((a.zout == nullptr) == (a.zout32 == nullptr) || a.dst != nullptr || a.src == nullptr)
+    return cudaErrorNotSupported;
   if (a.d % kUmmaCols != 0 || a.k > 128 || a.n < 4 * kUmmaTile || a.n > 0x7fffffffLL)
     return cudaErrorNotSupported;
   // a term with a prepared table is subtracted in the epilogue and needs no operand
@@ -486,6 +487,7 @@ cudaError_t launch_codec_mma(const MmaArgs &a, bool shift, int mode, int sm_coun
     cudaError_t e = launch_codec_umma_project(a, shift, sm_count, stream);
     if (e != cudaErrorNotSupported) return e;
   }
+  if (a.zout32 != nullptr) return cudaErrorNotSupported;   // wire rows: only the tcgen05 projection stores them
   if (mode == (kModeProject | kModeExpand) && !shift) {
     cudaError_t e = launch_codec_umma_roundtrip(a, sm_count, stream);
     if (e != cudaErrorNotSupported) return e;

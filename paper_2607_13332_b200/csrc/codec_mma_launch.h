@@ -23,6 +23,11 @@ struct MmaArgs {
   const __nv_bfloat16 *B1;
   int64_t ldb1;
   int32_t d1;
+  // projection with wire rows: the coordinates are stored as fp32 words in zout32 (zout is
+  // nullptr then); wire_ids != nullptr: word k of row t is wire_ids[t]
+  float *zout32;
+  int64_t ldzout32;
+  const int32_t *wire_ids;
   ShiftTables shift;
 };
 

@@ -524,6 +524,25 @@ codec_umma_project_kernel(const MmaArgs a, const __grid_constant__ UmmaMaps maps
           const int64_t pr = position_row(a.shift, t);
           if (pr >= 0) subtract_row(a.shift.PU + pr * a.shift.ldpu);
         }
+        if (a.zout32 != nullptr) {   // wire row: fp32 coordinates, then the token id
+          float *wrow = a.zout32 + t * a.ldzout32;
+          const bool vec4 = ((a.ldzout32 & 3) == 0) && ((reinterpret_cast<uintptr_t>(a.zout32) & 15) == 0);
+#pragma unroll
+          for (int q = 0; q < Cfg::kN / 16; ++q)
+#pragma unroll
+            for (int i = 0; i < 16; i += 4) {
+              const int col = q * 16 + i;
+              if (vec4 && col + 4 <= a.k) {
+                *reinterpret_cast<uint4 *>(wrow + col) = make_uint4(v[q][i], v[q][i + 1], v[q][i + 2], v[q][i + 3]);
+              } else {
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+                  if (col + e < a.k) wrow[col + e] = __uint_as_float(v[q][i + e]);
+              }
+            }
+          if (a.wire_ids != nullptr) reinterpret_cast<int32_t *>(wrow)[a.k] = a.wire_ids[t];
+          continue;
+        }
         __nv_bfloat16 *zrow = a.zout + t * a.ldzout;
 #pragma unroll
         for (int q = 0; q < Cfg::kN / 16; ++q) {

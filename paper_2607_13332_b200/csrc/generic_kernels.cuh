@@ -19,6 +19,10 @@ struct TokenArgs {
   const void *U2;     // expansion factor [d2 x k] when it differs from U (Eq. reparam), else nullptr
   int64_t ldu2;
   int32_t d2;
+  // wire rows (the bandwidth estimate of Sec. 3.5 counts the boundary tensors in FP32): the
+  // coordinates leave (zout, when projecting) or arrive (zin, when expanding) as fp32 words,
+  // leading dimension in words; with wire_ids word k of an outgoing row is the token id
+  int32_t wire, wire_ids;
   int32_t sub_shift;  // phase 1 subtracts E[ids]+P[pos]   (Eq. ssn_compress)
   int32_t add_shift;  // phase 2 adds E[ids]+P[pos] back   (receiver side)
   ShiftTables shift;
@@ -71,10 +75,18 @@ token_kernel(const TokenArgs a) {
       }
     }
     __syncwarp();
-    if (a.zout != nullptr) {
+    if (a.zout != nullptr && a.wire) {
+      float *z = static_cast<float *>(a.zout) + t * a.ldzout;
+      for (int j = lane; j < a.k; j += 32) z[j] = zs[j];
+      if (a.wire_ids && lane == 0) reinterpret_cast<int32_t *>(z)[a.k] = a.shift.ids[t];
+    } else if (a.zout != nullptr) {
       T *z = static_cast<T *>(a.zout) + t * a.ldzout;
       for (int j = lane; j < a.k; j += 32) z[j] = from_f32<T>(zs[j]);
     }
+  } else if (a.wire) {
+    const float *z = static_cast<const float *>(a.zin) + t * a.ldzin;
+    for (int j = lane; j < a.k; j += 32) zs[j] = z[j];
+    __syncwarp();
   } else {
     const T *z = static_cast<const T *>(a.zin) + t * a.ldzin;
     for (int j = lane; j < a.k; j += 32) zs[j] = to_f32(z[j]);
@@ -118,6 +130,49 @@ __global__ void gather_rows_kernel(const GatherArgs a) {
   T v = from_f32<T>(0.f);
   if (j < a.k && id >= 0 && id < a.rows) v = static_cast<const T *>(a.table)[id * a.ld_table + j];
   static_cast<T *>(a.out)[t * a.ld_out + j] = v;
+}
+
+// ---- wire rows in: ids out of word k, coordinates as bf16 head + remainder -------------------
+struct WireSplitArgs {
+  const float *wire;        // [n x ldw] words
+  __nv_bfloat16 *split;     // [n x 2 kp] or nullptr: head in columns [0, k), remainder in [kp, kp + k), zeros elsewhere
+  int32_t *ids;             // [n] or nullptr: word k of every row
+  int64_t ldw, n;
+  int32_t k, kp;
+};
+
+static __global__ void wire_split_kernel(const WireSplitArgs a) {
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const int w = a.split != nullptr ? a.kp : 1;     // threads per row
+  if (i >= a.n * w) return;
+  const int64_t t = i / w;
+  const int j = (int)(i - t * w);
+  const float *row = a.wire + t * a.ldw;
+  if (a.ids != nullptr && j == 0) a.ids[t] = reinterpret_cast<const int32_t *>(row)[a.k];
+  if (a.split != nullptr) {
+    const float z = j < a.k ? row[j] : 0.f;
+    const __nv_bfloat16 head = __float2bfloat16_rn(z);
+    a.split[t * 2 * a.kp + j] = head;
+    a.split[t * 2 * a.kp + a.kp + j] = __float2bfloat16_rn(z - __bfloat162float(head));
+  }
+}
+
+// U2 [d x 2 kp] = [U 0 | U 0]: the basis twice, so that (head | remainder) U2^T = (head + remainder) U^T
+struct BasisDupArgs {
+  const __nv_bfloat16 *U;
+  __nv_bfloat16 *U2;
+  int64_t ldu;
+  int32_t d, k, kp;
+};
+
+static __global__ void basis_dup_kernel(const BasisDupArgs a) {
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= (int64_t)a.d * a.kp) return;
+  const int64_t r = i / a.kp;
+  const int j = (int)(i - r * a.kp);
+  const __nv_bfloat16 v = j < a.k ? a.U[r * a.ldu + j] : __float2bfloat16_rn(0.f);
+  a.U2[r * 2 * a.kp + j] = v;
+  a.U2[r * 2 * a.kp + a.kp + j] = v;
 }
 
 // ---- contraction over tokens: out [m x k] (fp32) = H^T C, H [n x m], C [n x k] ---------------

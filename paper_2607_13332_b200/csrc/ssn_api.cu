@@ -113,13 +113,21 @@ ssn_status_t launch_generic_token_kernel(const TokenArgs &a, int32_t dtype, cuda
 
 ssn_status_t launch_token_kernel(const TokenArgs &a, int32_t dtype, cudaStream_t stream) {
   if (a.n == 0) return SSN_OK;
-  if (mma_eligible(a, dtype)) {
+  // wire rows: the tensor-core path takes the projection only (and falls back when it refuses)
+  const bool wire_ok = !a.wire || (a.src != nullptr && a.dst == nullptr);
+  if (wire_ok && mma_eligible(a, dtype)) {
     const int sms = sm_count_of_current_device();
     if (sms > 0) {
       MmaArgs m{};
       m.src = static_cast<const __nv_bfloat16 *>(a.src);
       m.zin = static_cast<const __nv_bfloat16 *>(a.zin);
-      m.zout = static_cast<__nv_bfloat16 *>(a.zout);
+      if (a.wire) {
+        m.zout32 = static_cast<float *>(a.zout);
+        m.ldzout32 = a.ldzout;
+        m.wire_ids = a.wire_ids ? a.shift.ids : nullptr;
+      } else {
+        m.zout = static_cast<__nv_bfloat16 *>(a.zout);
+      }
       m.dst = static_cast<__nv_bfloat16 *>(a.dst);
       m.U = static_cast<const __nv_bfloat16 *>(a.U);
       m.lds = a.lds;
@@ -134,8 +142,10 @@ ssn_status_t launch_token_kernel(const TokenArgs &a, int32_t dtype, cudaStream_t
       const bool shift = (a.sub_shift || a.add_shift) && (a.shift.E || a.shift.P);
       const int mode = (a.src ? 1 : 0) | (a.dst ? 2 : 0);
       cudaError_t e = launch_codec_mma(m, shift, mode, sms, stream);
-      g_launches.fetch_add(1, std::memory_order_relaxed);
-      return e == cudaSuccess ? SSN_OK : SSN_ERR_CUDA;
+      if (!(a.wire && e == cudaErrorNotSupported)) {
+        g_launches.fetch_add(1, std::memory_order_relaxed);
+        return e == cudaSuccess ? SSN_OK : SSN_ERR_CUDA;
+      }
     }
   }
   return launch_generic_token_kernel(a, dtype, stream);
@@ -404,6 +414,153 @@ ssn_status_t ssn_grad_project(const ssn_codec_t *codec, const void *G, int64_t l
   a.d = codec->d;
   a.k = codec->k;
   return launch_token_kernel(a, codec->dtype, static_cast<cudaStream_t>(stream));
+}
+
+// ---- wire rows ------------------------------------------------------------------------------
+namespace {
+inline size_t round256(size_t b) { return (b + 255) & ~(size_t)255; }
+inline int32_t padded_rank(int32_t k) { return (k + 7) & ~7; }
+// the tensor-core kernels take the fp32 coordinates as (head | remainder) of rank 2 * padded k
+inline bool wire_split_fits(const ssn_codec_t *c) { return c->dtype == SSN_BF16 && 2 * padded_rank(c->k) <= 128; }
+}  // namespace
+
+ssn_status_t ssn_compress_wire(const ssn_codec_t *codec, const void *X, int64_t ldx,
+                               const int32_t *ids, const int32_t *pos, int64_t n_tokens,
+                               int32_t seq_len, void *wire, int64_t ldw, int32_t with_ids,
+                               int32_t *dev_status, void *stream) {
+  ssn_status_t st = check_codec(codec);
+  if (st != SSN_OK) return st;
+  if (n_tokens < 0 || ldx < codec->d || ldw < (int64_t)codec->k + (with_ids ? 1 : 0)) return SSN_ERR_SHAPE;
+  if (with_ids && ids == nullptr) return SSN_ERR_NULL;
+  if (n_tokens == 0) return SSN_OK;
+  if (X == nullptr || wire == nullptr) return SSN_ERR_NULL;
+  TokenArgs a{};
+  st = make_shift(codec, ids, pos, seq_len, dev_status, &a.shift);
+  if (st != SSN_OK) return st;
+  a.src = X;
+  a.lds = ldx;
+  a.zout = wire;
+  a.ldzout = ldw;
+  a.wire = 1;
+  a.wire_ids = with_ids ? 1 : 0;
+  a.U = codec->U;
+  a.ldu = codec->ldu;
+  a.n = n_tokens;
+  a.d = codec->d;
+  a.k = codec->k;
+  a.sub_shift = 1;
+  if (codec->E != nullptr && codec->EU != nullptr) {
+    if (codec->ldeu < codec->k) return SSN_ERR_SHAPE;
+    a.shift.EU = codec->EU;
+    a.shift.ldeu = codec->ldeu;
+  }
+  if (codec->P != nullptr && codec->PU != nullptr) {
+    if (codec->ldpu < codec->k) return SSN_ERR_SHAPE;
+    a.shift.PU = codec->PU;
+    a.shift.ldpu = codec->ldpu;
+  }
+  return launch_token_kernel(a, codec->dtype, static_cast<cudaStream_t>(stream));
+}
+
+ssn_status_t ssn_grad_project_wire(const ssn_codec_t *codec, const void *G, int64_t ldg,
+                                   int64_t n_tokens, float *dZ, int64_t ldw, void *stream) {
+  ssn_status_t st = check_codec(codec);
+  if (st != SSN_OK) return st;
+  if (n_tokens < 0 || ldg < codec->d || ldw < codec->k) return SSN_ERR_SHAPE;
+  if (n_tokens == 0) return SSN_OK;
+  if (G == nullptr || dZ == nullptr) return SSN_ERR_NULL;
+  TokenArgs a{};
+  a.src = G;
+  a.lds = ldg;
+  a.zout = dZ;
+  a.ldzout = ldw;
+  a.wire = 1;
+  a.U = codec->U;
+  a.ldu = codec->ldu;
+  a.n = n_tokens;
+  a.d = codec->d;
+  a.k = codec->k;
+  return launch_token_kernel(a, codec->dtype, static_cast<cudaStream_t>(stream));
+}
+
+size_t ssn_decompress_wire_workspace_bytes(const ssn_codec_t *codec, int64_t n_tokens, int32_t with_ids) {
+  if (check_codec(codec) != SSN_OK || n_tokens < 0) return 0;
+  size_t bytes = with_ids ? round256((size_t)n_tokens * sizeof(int32_t)) : 0;
+  if (wire_split_fits(codec)) {
+    const size_t kp2 = 2 * (size_t)padded_rank(codec->k);
+    bytes += round256((size_t)n_tokens * kp2 * 2) + round256((size_t)codec->d * kp2 * 2);
+  }
+  return bytes;
+}
+
+ssn_status_t ssn_decompress_wire(const ssn_codec_t *codec, const void *wire, int64_t ldw,
+                                 int32_t with_ids, const int32_t *ids, const int32_t *pos,
+                                 int64_t n_tokens, int32_t seq_len, void *Xhat, int64_t ldx,
+                                 void *workspace, size_t workspace_bytes, int32_t *dev_status,
+                                 void *stream) {
+  ssn_status_t st = check_codec(codec);
+  if (st != SSN_OK) return st;
+  if (n_tokens < 0 || ldx < codec->d || ldw < (int64_t)codec->k + (with_ids ? 1 : 0)) return SSN_ERR_SHAPE;
+  if (n_tokens == 0) return SSN_OK;
+  if (Xhat == nullptr || wire == nullptr) return SSN_ERR_NULL;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const size_t ids_bytes = with_ids ? round256((size_t)n_tokens * sizeof(int32_t)) : 0;
+  if (with_ids && (workspace == nullptr || workspace_bytes < ids_bytes)) return SSN_ERR_WORKSPACE;
+  unsigned char *ws = static_cast<unsigned char *>(workspace);
+  int32_t *ids_out = with_ids ? reinterpret_cast<int32_t *>(ws) : nullptr;
+  const int32_t kp = padded_rank(codec->k);
+  const size_t split_bytes = round256((size_t)n_tokens * 2 * kp * 2), u2_bytes = round256((size_t)codec->d * 2 * kp * 2);
+  const bool split = wire_split_fits(codec) && workspace != nullptr && (reinterpret_cast<uintptr_t>(workspace) & 255) == 0 &&
+                     workspace_bytes >= ids_bytes + split_bytes + u2_bytes;
+  WireSplitArgs w{};
+  w.wire = static_cast<const float *>(wire);
+  w.ldw = ldw;
+  w.n = n_tokens;
+  w.k = codec->k;
+  w.kp = kp;
+  w.ids = ids_out;
+  w.split = split ? reinterpret_cast<__nv_bfloat16 *>(ws + ids_bytes) : nullptr;
+  if (w.ids != nullptr || w.split != nullptr) {
+    const int64_t threads = n_tokens * (split ? kp : 1), blocks = (threads + 255) / 256;
+    if (blocks > 0x7fffffffLL) return SSN_ERR_SHAPE;
+    wire_split_kernel<<<(unsigned)blocks, 256, 0, s>>>(w);
+    st = launch_status();
+    if (st != SSN_OK) return st;
+  }
+  TokenArgs a{};
+  st = make_shift(codec, with_ids ? ids_out : ids, pos, seq_len, dev_status, &a.shift);
+  if (st != SSN_OK) return st;
+  a.dst = Xhat;
+  a.lddst = ldx;
+  a.n = n_tokens;
+  a.d = codec->d;
+  a.add_shift = 1;
+  if (split) {
+    BasisDupArgs b{};
+    b.U = static_cast<const __nv_bfloat16 *>(codec->U);
+    b.U2 = reinterpret_cast<__nv_bfloat16 *>(ws + ids_bytes + split_bytes);
+    b.ldu = codec->ldu;
+    b.d = codec->d;
+    b.k = codec->k;
+    b.kp = kp;
+    const int64_t blocks = ((int64_t)codec->d * kp + 255) / 256;
+    basis_dup_kernel<<<(unsigned)blocks, 256, 0, s>>>(b);
+    st = launch_status();
+    if (st != SSN_OK) return st;
+    a.zin = w.split;
+    a.ldzin = 2 * kp;
+    a.U = b.U2;
+    a.ldu = 2 * kp;
+    a.k = 2 * kp;
+  } else {
+    a.zin = wire;
+    a.ldzin = ldw;
+    a.wire = 1;
+    a.U = codec->U;
+    a.ldu = codec->ldu;
+    a.k = codec->k;
+  }
+  return launch_token_kernel(a, codec->dtype, s);
 }
 
 ssn_status_t ssn_reparam_project(const ssn_codec_t *codec, const void *H, int64_t ldh, int64_t m,

@@ -135,6 +135,47 @@ class Codec:
             return dZ, Gp
         return dZ if coeff else Gp
 
+    # ---- wire rows: k fp32 coordinates (+ the token id as an int32 word) per token ------------
+    def wire_buffer(self, n: int, with_ids: bool, ldw: Optional[int] = None) -> torch.Tensor:
+        """An int32-typed [n, ldw] buffer of wire words (view the coordinates with .view(torch.float32))."""
+        ldw = ldw if ldw is not None else self.k + (1 if with_ids else 0)
+        return torch.empty((n, ldw), dtype=torch.int32, device=self.U.device)
+
+    def compress_wire(self, X: torch.Tensor, ids: Optional[torch.Tensor] = None, seq_len: int = 1,
+                      pos: Optional[torch.Tensor] = None, with_ids: bool = False,
+                      out: Optional[torch.Tensor] = None) -> torch.Tensor:
+        n = X.shape[0]
+        wire = out if out is not None else self.wire_buffer(n, with_ids)
+        binding.ssn_compress_wire(self.c, X.data_ptr(), _ld(X), ids.data_ptr() if ids is not None else 0,
+                                  pos.data_ptr() if pos is not None else 0, n, seq_len, wire.data_ptr(),
+                                  _ld(wire), with_ids, self.dev_status.data_ptr(), _stream())
+        return wire
+
+    def grad_project_wire(self, G: torch.Tensor, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+        n = G.shape[0]
+        dZ = out if out is not None else torch.empty((n, self.k), dtype=torch.float32, device=self.U.device)
+        binding.ssn_grad_project_wire(self.c, G.data_ptr(), _ld(G), n, dZ.data_ptr(), _ld(dZ), _stream())
+        return dZ
+
+    def decompress_wire(self, wire: torch.Tensor, ids: Optional[torch.Tensor] = None, seq_len: int = 1,
+                        pos: Optional[torch.Tensor] = None, with_ids: bool = False,
+                        out: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None,
+                        use_workspace: bool = True) -> torch.Tensor:
+        n = wire.shape[0]
+        Xh = out if out is not None else self._empty(n, self.d)
+        if workspace is None:
+            nbytes = binding.ssn_decompress_wire_workspace_bytes(self.c, n, with_ids)
+            if not use_workspace:   # only what the ids need: the general kernel runs
+                nbytes = (n * 4 + 255) // 256 * 256 if with_ids else 0
+            workspace = torch.empty(nbytes, dtype=torch.uint8, device=self.U.device) if nbytes else None
+        binding.ssn_decompress_wire(self.c, wire.data_ptr(), _ld(wire), with_ids,
+                                    ids.data_ptr() if ids is not None else 0,
+                                    pos.data_ptr() if pos is not None else 0, n, seq_len, Xh.data_ptr(), _ld(Xh),
+                                    workspace.data_ptr() if workspace is not None else 0,
+                                    workspace.numel() if workspace is not None else 0,
+                                    self.dev_status.data_ptr(), _stream())
+        return Xh
+
     def reproject_workspace(self, rows: int, cols: int, side: str, batch: int) -> Optional[torch.Tensor]:
         nbytes = binding.ssn_weight_reproject_workspace_bytes(self.c, rows, cols, binding.SIDES[side], batch)
         if nbytes == 0:

@@ -419,3 +419,28 @@ def test_head_embed_is_gather_of_the_materialised_table_and_is_recovered_by_comp
     X1, status = oracle.head_embed(Elow, U, E, bad, P, pos)
     assert status == oracle.STATUS_BAD_ID and np.abs(X1[2] - P[pos[2]]).max() == 0.0
 
+
+
+# ---- wire rows -------------------------------------------------------------------------------
+def test_wire_rows_bit_patterns():
+    """IEEE-754 single patterns typed by hand: 1.0, -2.5, 0.1 (rounds to 0x3DCCCCCD), 0; the id word."""
+    Z = np.array([[1.0, -2.5], [0.1, 0.0]])
+    w = oracle.wire_rows(Z, ids=[7, 128255])
+    assert w.dtype == np.int32 and w.shape == (2, 3)
+    as_u32 = w.view(np.uint32)
+    assert as_u32[0, 0] == 0x3F800000 and as_u32[0, 1] == 0xC0200000
+    assert as_u32[1, 0] == 0x3DCCCCCD and as_u32[1, 1] == 0
+    assert w[0, 2] == 7 and w[1, 2] == 128255
+    assert oracle.wire_rows(Z).shape == (2, 2)
+
+
+def test_wire_round_trip_half_ulp():
+    rng = np.random.default_rng(5)
+    Z = rng.standard_normal((37, 11)) * np.exp(rng.uniform(-20, 20, size=(37, 11)))
+    ids = rng.integers(0, 2 ** 31 - 1, size=37)
+    back, ids_back = oracle.wire_unpack(oracle.wire_rows(Z, ids), 11, True)
+    assert np.array_equal(ids_back, ids)
+    assert np.all(np.abs(back - Z) <= np.abs(Z) * 2.0 ** -24)
+    # values that are float32 already travel unchanged
+    Z32 = Z.astype(np.float32).astype(np.float64)
+    assert np.array_equal(oracle.wire_unpack(oracle.wire_rows(Z32), 11, False)[0], Z32)
