@@ -496,7 +496,8 @@ def run_sweep(args):
         E = (torch.randn((vocab, d), device="cuda", generator=gen) * 0.02).bfloat16()
         P = to_device(synth.to_storage(synth.sinusoidal_positions(seq, d), dt), dt)
         X = torch.randn((n, d), device="cuda", generator=gen).bfloat16()
-        Xh = torch.empty_like(X)
+        Xh = torch.randn((n, d), device="cuda", generator=gen).bfloat16()
+        Xs = torch.empty_like(X)
         for k in (24, 40):
             U = to_device(synth.to_storage(synth.subspace_basis(d, k, 1), dt), dt)
             codec, codec_t = Codec(dt, U, E, P), Codec(dt, U, E, P)
@@ -514,6 +515,13 @@ def run_sweep(args):
                  lambda: codec_t.compress_wire(X, ids, seq_len=seq, with_ids=True, out=wire),
                  n * d * 2 + n * 4 + (uniq + seq) * k * 4 + d * k * 2 + n * (k + 1) * 4),
                 ("compress (bf16 rows)", lambda: codec.compress(X, ids, seq_len=seq, out=Z), rows_in + n * k * 2),
+                # the stage's last residual add fused in (X + R is never written): two reads of n x d
+                ("compress_sum -> wire rows, prepared tables",
+                 lambda: codec_t.compress_sum(X, Xh, ids, seq_len=seq, wire=True, with_ids=True, out=wire),
+                 2 * n * d * 2 + n * 4 + (uniq + seq) * k * 4 + d * k * 2 + n * (k + 1) * 4),
+                ("unfused: torch add, then compress_wire with prepared tables (same algorithmic bytes)",
+                 lambda: codec_t.compress_wire(torch.add(X, Xh, out=Xs), ids, seq_len=seq, with_ids=True, out=wire),
+                 2 * n * d * 2 + n * 4 + (uniq + seq) * k * 4 + d * k * 2 + n * (k + 1) * 4),
                 ("grad_project_wire", lambda: codec.grad_project_wire(X, out=dZ), n * d * 2 + d * k * 2 + n * k * 4),
                 ("decompress_wire",
                  lambda: codec.decompress_wire(wire, seq_len=seq, with_ids=True, out=Xh, workspace=ws),

@@ -281,6 +281,25 @@ ssn_status_t ssn_decompress_wire(const ssn_codec_t *codec, const void *wire, int
                                  void *stream);
 
 /*
+ * Compress fused with the stage's last residual add (Eq. residual_stream: the hidden state that
+ * reaches the boundary is the residual stream plus the last block's output; Eq. ssn_compress):
+ *     Z = (X + R - P[pos] - E[ids]) U
+ * X and R are [n x d] in the storage dtype (leading dimensions ldx, ldr >= d); their sum is never
+ * formed in memory nor rounded to the storage dtype.  out_form selects what is written:
+ *   SSN_OUT_STORAGE   Z [n x k] in the storage dtype, ldout >= k elements   (as ssn_compress)
+ *   SSN_OUT_WIRE      wire rows, ldout >= k words                          (as ssn_compress_wire)
+ *   SSN_OUT_WIRE_IDS  wire rows with the id word, ldout >= k + 1 words
+ * Everything else as for ssn_compress.  Performance note: the tensor-core kernel takes this call
+ * for a codec without E and P or with the prepared tables (ssn_prepare_tables); a codec that has
+ * to gather E or P rows runs the general kernel here.
+ */
+enum { SSN_OUT_STORAGE = 0, SSN_OUT_WIRE = 1, SSN_OUT_WIRE_IDS = 2 };
+ssn_status_t ssn_compress_sum(const ssn_codec_t *codec, const void *X, int64_t ldx, const void *R,
+                              int64_t ldr, const int32_t *ids, const int32_t *pos, int64_t n_tokens,
+                              int32_t seq_len, void *out, int64_t ldout, int32_t out_form,
+                              int32_t *dev_status, void *stream);
+
+/*
  * LEFT re-projection of ONE weight, W [d x cols] <- U (U^T W), without a caller workspace.
  * (The paper has no counterpart: this is a packaging variant of ssn_weight_reproject.)
  *

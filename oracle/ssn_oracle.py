@@ -25,7 +25,8 @@ gather, isometry at k = d, exact round trip inside the subspace, adjoint and fin
 identities, projector identities, explicit d x d projector, element-by-element loops on tiny
 shapes; for the reparameterized forms (Eq. reparam): the materialised weight W_p = Z U^T, its
 membership of the subspace, loops, and the exact recovery of the factored embedding's coordinates
-by compress; for the wire rows: IEEE-754 bit patterns typed by hand, the id word, the round trip
+by compress; for compress_sum: linearity against a loop-written R U and the exact recovery of
+summed coordinates; for the wire rows: IEEE-754 bit patterns typed by hand, the id word, the round trip
 within half an fp32 ulp.  No function here is left unpinned.
 """
 
@@ -74,6 +75,16 @@ def compress(X: np.ndarray, U: np.ndarray, E=None, ids=None, P=None, pos=None):
     U = np.asarray(U, dtype=np.float64)
     shift, status = shift_rows(X.shape[0], X.shape[1], E, ids, P, pos)
     return (X - shift) @ U, status
+
+
+def compress_sum(X: np.ndarray, R: np.ndarray, U: np.ndarray, E=None, ids=None, P=None, pos=None):
+    """Eq. ssn_compress applied to the hidden state of Eq. residual_stream written as residual stream
+    plus the last block's output, X + R, the sum exact (float64).  Returns (Z [n, k], status)."""
+    X = np.asarray(X, dtype=np.float64)
+    R = np.asarray(R, dtype=np.float64)
+    U = np.asarray(U, dtype=np.float64)
+    shift, status = shift_rows(X.shape[0], X.shape[1], E, ids, P, pos)
+    return ((X + R) - shift) @ U, status
 
 
 def decompress(Z: np.ndarray, U: np.ndarray, E=None, ids=None, P=None, pos=None):

@@ -71,6 +71,7 @@ _SIGNATURES = {
     "ssn_reparam_grad_factor": (_i32, [_codec_p, _vp, _i64, _i64, _vp, _i64, _i64, _vp, _i64, _vp, _sz, _vp]),
     "ssn_head_embed": (_i32, [_codec_p, _vp, _i64, _i64, _vp, _vp, _i64, _i32, _vp, _i64, _vp, _sz, _vp, _vp]),
     "ssn_compress_wire": (_i32, [_codec_p, _vp, _i64, _vp, _vp, _i64, _i32, _vp, _i64, _i32, _vp, _vp]),
+    "ssn_compress_sum": (_i32, [_codec_p, _vp, _i64, _vp, _i64, _vp, _vp, _i64, _i32, _vp, _i64, _i32, _vp, _vp]),
     "ssn_grad_project_wire": (_i32, [_codec_p, _vp, _i64, _i64, _vp, _i64, _vp]),
     "ssn_decompress_wire_workspace_bytes": (_sz, [_codec_p, _i64, _i32]),
     "ssn_decompress_wire": (_i32, [_codec_p, _vp, _i64, _i32, _vp, _vp, _i64, _i32, _vp, _i64, _vp, _sz,
@@ -213,6 +214,18 @@ def ssn_compress_wire(codec: ssn_codec_t, X: int, ldx: int, ids: int, pos: int, 
     _check(_lib.ssn_compress_wire(ctypes.byref(codec), X or None, ldx, ids or None, pos or None, n_tokens,
                                   seq_len, wire or None, ldw, 1 if with_ids else 0, dev_status or None,
                                   stream or None), "ssn_compress_wire")
+
+
+SSN_OUT_STORAGE, SSN_OUT_WIRE, SSN_OUT_WIRE_IDS = 0, 1, 2
+
+
+def ssn_compress_sum(codec: ssn_codec_t, X: int, ldx: int, R: int, ldr: int, ids: int, pos: int, n_tokens: int,
+                     seq_len: int, out: int, ldout: int, out_form: int = SSN_OUT_STORAGE, dev_status: int = 0,
+                     stream: int = 0) -> None:
+    """Z = (X + R - P[pos] - E[ids]) U: compress fused with the stage's last residual add."""
+    _check(_lib.ssn_compress_sum(ctypes.byref(codec), X or None, ldx, R or None, ldr, ids or None, pos or None,
+                                 n_tokens, seq_len, out or None, ldout, out_form, dev_status or None,
+                                 stream or None), "ssn_compress_sum")
 
 
 def ssn_grad_project_wire(codec: ssn_codec_t, G: int, ldg: int, n_tokens: int, dZ: int, ldw: int,

@@ -264,6 +264,11 @@ cudaError_t launch_codec_umma_project(const MmaArgs &a, bool shift, int sm_count
   if (!make_sw128_map(&maps.u_wide, a.U, a.d, a.k <= 64 ? 64 : 128, a.ldu, kUmmaCols))
     return cudaErrorNotSupported;
   maps.p = maps.x;
+  maps.x2 = maps.x;
+  if (a.src2 != nullptr) {   // a second addend: only the launches without row operands take it
+    if (has_e || has_p) return cudaErrorNotSupported;
+    if (!make_sw128_map(&maps.x2, a.src2, a.n, a.d, a.lds2, kUmmaTile)) return cudaErrorNotSupported;
+  }
   if (has_p && !make_sw128_map(&maps.p, a.shift.P, a.shift.max_pos, a.d, a.shift.ldp, kUmmaTile))
     return cudaErrorNotSupported;
   if (ntp <= 2) return launch_umma_ntp<2>(b, has_e, has_p, maps, sm_count, stream);
@@ -487,7 +492,8 @@ cudaError_t launch_codec_mma(const MmaArgs &a, bool shift, int mode, int sm_coun
     cudaError_t e = launch_codec_umma_project(a, shift, sm_count, stream);
     if (e != cudaErrorNotSupported) return e;
   }
-  if (a.zout32 != nullptr) return cudaErrorNotSupported;   // wire rows: only the tcgen05 projection stores them
+  // wire rows and a second addend: only the tcgen05 projection takes them
+  if (a.zout32 != nullptr || a.src2 != nullptr) return cudaErrorNotSupported;
   if (mode == (kModeProject | kModeExpand) && !shift) {
     cudaError_t e = launch_codec_umma_roundtrip(a, sm_count, stream);
     if (e != cudaErrorNotSupported) return e;

@@ -23,6 +23,10 @@ struct MmaArgs {
   const __nv_bfloat16 *B1;
   int64_t ldb1;
   int32_t d1;
+  // projection of a sum (the stage's last residual add fused into compress): Z = (src + src2) U,
+  // tcgen05 projection without row operands only; nullptr: none
+  const __nv_bfloat16 *src2;
+  int64_t lds2;
   // projection with wire rows: the coordinates are stored as fp32 words in zout32 (zout is
   // nullptr then); wire_ids != nullptr: word k of row t is wire_ids[t]
   float *zout32;

@@ -165,8 +165,11 @@ struct UmmaProjectConfig {
 // row pitch, so that a box never leaves the tensor: the columns past k then hold the start of
 // the following rows, and feed only accumulator columns that are never stored.  u_wide is used
 // for all stages but the last one of U, whose box would read past the end of the buffer.
+// x2: a second matrix of rows to project with the same tiles (a.src2 != nullptr): the
+// contraction then runs over the columns of x and, after them, over the columns of x2 against
+// the same slices of U, i.e. Z = (X + X2) U with the sum never formed or rounded.
 struct UmmaMaps {
-  CUtensorMap x, p, u, u_wide;
+  CUtensorMap x, p, u, u_wide, x2;
 };
 
 template <int NTP, bool HAS_E, bool HAS_P>
@@ -177,7 +180,8 @@ codec_umma_project_kernel(const MmaArgs a, const __grid_constant__ UmmaMaps maps
   constexpr int S = Cfg::kStagesN;
   extern __shared__ __align__(128) unsigned char smem_raw[];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int nstage = a.d / kUmmaCols;
+  const int nstage1 = a.d / kUmmaCols;                                  // stages of one matrix
+  const int nstage = (!HAS_E && !HAS_P && a.src2 != nullptr) ? 2 * nstage1 : nstage1;
   const int64_t ntiles = (a.n + kUmmaTile - 1) / kUmmaTile;
 
   const uint32_t smem0 = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -300,12 +304,13 @@ codec_umma_project_kernel(const MmaArgs a, const __grid_constant__ UmmaMaps maps
         const uint32_t bar = full_bar(slot);
         if (lane == 0) {
           mbar_expect_tx(bar, Cfg::kTmaBytes - (HAS_P && !load_p ? Cfg::kATileBytes : 0));
-          tma_load_2d(base, &maps.x, bar, st * kUmmaCols, (int)tok0);
+          const int su = st < nstage1 ? st : st - nstage1;   // slice of U; the second matrix starts over
+          tma_load_2d(base, st < nstage1 ? &maps.x : &maps.x2, bar, su * kUmmaCols, (int)tok0);
           if (load_p) tma_load_2d(base + kPTile * Cfg::kATileBytes, &maps.p, bar, st * kUmmaCols, pos0);
 #pragma unroll
           for (int ug = 0; ug < Cfg::kUGroups; ++ug)
             tma_load_2d(base + Cfg::kATiles * Cfg::kATileBytes + ug * Cfg::kUGroupBytes,
-                        st == nstage - 1 ? &maps.u : &maps.u_wide, bar, ug * 64, st * kUmmaCols);
+                        su == nstage1 - 1 ? &maps.u : &maps.u_wide, bar, ug * 64, su * kUmmaCols);
         }
         __syncwarp();
         if (++slot == S) {

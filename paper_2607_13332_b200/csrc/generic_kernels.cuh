@@ -9,6 +9,8 @@ namespace ssn {
 
 struct TokenArgs {
   const void *src;   // [n x d] rows to project (X, G or W), or nullptr: read coordinates from zin
+  const void *src2;  // [n x d] second addend of the rows to project (projection only), or nullptr
+  int64_t lds2;
   const void *zin;   // [n x k] coordinates when src == nullptr
   void *zout;        // [n x k] coordinates out, nullable
   void *dst;         // [n x d] expansion out, nullable (may alias src row-for-row)
@@ -50,6 +52,7 @@ token_kernel(const TokenArgs a) {
 
   if (a.src != nullptr) {
     const T *x = static_cast<const T *>(a.src) + t * a.lds;
+    const T *x2 = a.src2 != nullptr ? static_cast<const T *>(a.src2) + t * a.lds2 : nullptr;
     for (int j0 = 0; j0 < a.k; j0 += kGenericKChunk) {
       float acc[kGenericKChunk];
 #pragma unroll
@@ -57,6 +60,7 @@ token_kernel(const TokenArgs a) {
       const int jn = min(kGenericKChunk, a.k - j0);
       for (int i = lane; i < a.d; i += 32) {
         float r = to_f32(x[i]);
+        if (x2 != nullptr) r += to_f32(x2[i]);
         if (a.sub_shift) {
           if (erow) r -= to_f32(erow[i]);
           if (prow) r -= to_f32(prow[i]);

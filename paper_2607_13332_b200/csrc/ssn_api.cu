@@ -78,6 +78,7 @@ bool mma_eligible(const TokenArgs &a, int32_t dtype) {
   if (dtype != SSN_BF16 || !codec_mma_supports(a.d, a.k)) return false;
   if (!aligned16(a.U) || (a.ldu & 7)) return false;
   if (a.src && (!aligned16(a.src) || (a.lds & 7))) return false;
+  if (a.src2 && (!aligned16(a.src2) || (a.lds2 & 7))) return false;
   if (a.dst && (!aligned16(a.dst) || (a.lddst & 7))) return false;
   if (a.sub_shift || a.add_shift) {
     if (a.shift.E && (!aligned16(a.shift.E) || (a.shift.lde & 7))) return false;
@@ -114,7 +115,7 @@ ssn_status_t launch_generic_token_kernel(const TokenArgs &a, int32_t dtype, cuda
 ssn_status_t launch_token_kernel(const TokenArgs &a, int32_t dtype, cudaStream_t stream) {
   if (a.n == 0) return SSN_OK;
   // wire rows: the tensor-core path takes the projection only (and falls back when it refuses)
-  const bool wire_ok = !a.wire || (a.src != nullptr && a.dst == nullptr);
+  const bool wire_ok = !(a.wire || a.src2) || (a.src != nullptr && a.dst == nullptr);
   if (wire_ok && mma_eligible(a, dtype)) {
     const int sms = sm_count_of_current_device();
     if (sms > 0) {
@@ -130,6 +131,8 @@ ssn_status_t launch_token_kernel(const TokenArgs &a, int32_t dtype, cudaStream_t
       }
       m.dst = static_cast<__nv_bfloat16 *>(a.dst);
       m.U = static_cast<const __nv_bfloat16 *>(a.U);
+      m.src2 = static_cast<const __nv_bfloat16 *>(a.src2);
+      m.lds2 = a.lds2;
       m.lds = a.lds;
       m.ldzin = a.ldzin;
       m.ldzout = a.ldzout;
@@ -142,7 +145,7 @@ ssn_status_t launch_token_kernel(const TokenArgs &a, int32_t dtype, cudaStream_t
       const bool shift = (a.sub_shift || a.add_shift) && (a.shift.E || a.shift.P);
       const int mode = (a.src ? 1 : 0) | (a.dst ? 2 : 0);
       cudaError_t e = launch_codec_mma(m, shift, mode, sms, stream);
-      if (!(a.wire && e == cudaErrorNotSupported)) {
+      if (!((a.wire || a.src2) && e == cudaErrorNotSupported)) {
         g_launches.fetch_add(1, std::memory_order_relaxed);
         return e == cudaSuccess ? SSN_OK : SSN_ERR_CUDA;
       }
@@ -442,6 +445,49 @@ ssn_status_t ssn_compress_wire(const ssn_codec_t *codec, const void *X, int64_t 
   a.zout = wire;
   a.ldzout = ldw;
   a.wire = 1;
+  a.wire_ids = with_ids ? 1 : 0;
+  a.U = codec->U;
+  a.ldu = codec->ldu;
+  a.n = n_tokens;
+  a.d = codec->d;
+  a.k = codec->k;
+  a.sub_shift = 1;
+  if (codec->E != nullptr && codec->EU != nullptr) {
+    if (codec->ldeu < codec->k) return SSN_ERR_SHAPE;
+    a.shift.EU = codec->EU;
+    a.shift.ldeu = codec->ldeu;
+  }
+  if (codec->P != nullptr && codec->PU != nullptr) {
+    if (codec->ldpu < codec->k) return SSN_ERR_SHAPE;
+    a.shift.PU = codec->PU;
+    a.shift.ldpu = codec->ldpu;
+  }
+  return launch_token_kernel(a, codec->dtype, static_cast<cudaStream_t>(stream));
+}
+
+ssn_status_t ssn_compress_sum(const ssn_codec_t *codec, const void *X, int64_t ldx, const void *R,
+                              int64_t ldr, const int32_t *ids, const int32_t *pos, int64_t n_tokens,
+                              int32_t seq_len, void *out, int64_t ldout, int32_t out_form,
+                              int32_t *dev_status, void *stream) {
+  ssn_status_t st = check_codec(codec);
+  if (st != SSN_OK) return st;
+  if (out_form != SSN_OUT_STORAGE && out_form != SSN_OUT_WIRE && out_form != SSN_OUT_WIRE_IDS) return SSN_ERR_DTYPE;
+  const bool with_ids = out_form == SSN_OUT_WIRE_IDS;
+  if (n_tokens < 0 || ldx < codec->d || ldr < codec->d || ldout < (int64_t)codec->k + (with_ids ? 1 : 0))
+    return SSN_ERR_SHAPE;
+  if (with_ids && ids == nullptr) return SSN_ERR_NULL;
+  if (n_tokens == 0) return SSN_OK;
+  if (X == nullptr || R == nullptr || out == nullptr) return SSN_ERR_NULL;
+  TokenArgs a{};
+  st = make_shift(codec, ids, pos, seq_len, dev_status, &a.shift);
+  if (st != SSN_OK) return st;
+  a.src = X;
+  a.lds = ldx;
+  a.src2 = R;
+  a.lds2 = ldr;
+  a.zout = out;
+  a.ldzout = ldout;
+  a.wire = out_form != SSN_OUT_STORAGE ? 1 : 0;
   a.wire_ids = with_ids ? 1 : 0;
   a.U = codec->U;
   a.ldu = codec->ldu;

@@ -151,6 +151,20 @@ class Codec:
                                   _ld(wire), with_ids, self.dev_status.data_ptr(), _stream())
         return wire
 
+    def compress_sum(self, X: torch.Tensor, R: torch.Tensor, ids: Optional[torch.Tensor] = None, seq_len: int = 1,
+                     pos: Optional[torch.Tensor] = None, wire: bool = False, with_ids: bool = False,
+                     out: Optional[torch.Tensor] = None) -> torch.Tensor:
+        """compress(X + R) without forming the sum; Z in the storage dtype, or wire rows."""
+        n = X.shape[0]
+        if out is None:
+            out = self.wire_buffer(n, with_ids) if wire else self._empty(n, self.k)
+        form = (binding.SSN_OUT_WIRE_IDS if with_ids else binding.SSN_OUT_WIRE) if wire else binding.SSN_OUT_STORAGE
+        binding.ssn_compress_sum(self.c, X.data_ptr(), _ld(X), R.data_ptr(), _ld(R),
+                                 ids.data_ptr() if ids is not None else 0,
+                                 pos.data_ptr() if pos is not None else 0, n, seq_len, out.data_ptr(), _ld(out),
+                                 form, self.dev_status.data_ptr(), _stream())
+        return out
+
     def grad_project_wire(self, G: torch.Tensor, out: Optional[torch.Tensor] = None) -> torch.Tensor:
         n = G.shape[0]
         dZ = out if out is not None else torch.empty((n, self.k), dtype=torch.float32, device=self.U.device)

@@ -136,3 +136,65 @@ def test_wire_argument_errors():
     assert binding.ssn_decompress_wire_workspace_bytes(codec.c, n, True) >= n * 4 + n * 16 * 2 + 128 * 16 * 2
     assert binding.ssn_decompress_wire_workspace_bytes(codec.c, n, False) > 0
     binding.ssn_compress_wire(codec.c, X.data_ptr(), 128, ids.data_ptr(), 0, 0, 64, 0, 9, True)   # empty batch
+
+
+# batch, seq_len, d, k, vocab, dtype
+SUM_CASES = [
+    (8, 128, 512, 40, 300, synth.BF16),
+    (9, 128, 1024, 64, 500, synth.BF16),     # odd tile count: a pair splits its last tile between X and R
+    (75, 128, 256, 16, 100, synth.BF16),     # more tiles than CTA pairs
+    (8, 128, 256, 96, 100, synth.BF16),      # two coordinate groups
+    (8, 128, 64, 8, 50, synth.BF16),         # one stage per matrix
+    (3, 50, 128, 5, 40, synth.BF16),         # few tokens: general kernel
+    (2, 64, 128, 8, 30, synth.F32),
+]
+
+
+@pytest.mark.parametrize("batch,seq_len,d,k,vocab,dt", SUM_CASES)
+def test_compress_sum(batch, seq_len, d, k, vocab, dt):
+    """Z = (X + R - E - P) U on a codec with prepared tables (tensor cores), with gathered rows
+    (general kernel) and without E and P, in the three output forms."""
+    wl = synth.Workload("sum", d, k, vocab, batch, seq_len, dt)
+    t = synth.codec_inputs(wl, seed=batch + d + k, noise_std=0.05)
+    n = wl.n_tokens
+    rng = np.random.default_rng(batch + k)
+    R0 = synth.to_storage(rng.standard_normal((n, d)) * 0.3, dt)
+    X, R = to_device(t["X"], dt), to_device(R0, dt)
+    ids = torch.from_numpy(t["ids"]).cuda()
+    pos = oracle.token_positions(n, seq_len)
+    Uf, Ef, Pf = f64(t["U"], dt), f64(t["E"], dt), f64(t["P"], dt)
+    expect, _ = oracle.compress_sum(f64(t["X"], dt), f64(R0, dt), Uf, Ef, t["ids"], Pf, pos)
+    rows = Codec(dt, to_device(t["U"], dt), to_device(t["E"], dt), to_device(t["P"], dt))
+    tables = Codec(dt, to_device(t["U"], dt), to_device(t["E"], dt), to_device(t["P"], dt))
+    tables.prepare_tables()
+    for name, codec in (("gathered rows", rows), ("prepared tables", tables)):
+        Z = codec.compress_sum(X, R, ids, seq_len=seq_len)
+        assert_close(host64(Z, dt), expect, dt, f"compress_sum, {name}")
+        w = codec.compress_sum(X, R, ids, seq_len=seq_len, wire=True, with_ids=True)
+        got, got_ids = oracle.wire_unpack(w.cpu().numpy(), k, True)
+        assert_close(got, expect, dt, f"compress_sum wire rows, {name}", tol=WIRE_TOL)
+        assert np.array_equal(got_ids, t["ids"])
+        assert codec.take_status() == 0
+    bare = Codec(dt, to_device(t["U"], dt))
+    w = bare.compress_sum(X, R, wire=True)
+    assert_close(oracle.wire_unpack(w.cpu().numpy(), k, False)[0],
+                 oracle.compress_sum(f64(t["X"], dt), f64(R0, dt), Uf)[0], dt, "compress_sum, no tables", tol=WIRE_TOL)
+    assert torch.equal(X, to_device(t["X"], dt)) and torch.equal(R, to_device(R0, dt))
+
+
+def test_compress_sum_argument_errors():
+    dt = synth.BF16
+    wl = synth.Workload("sum", 128, 8, 50, 2, 64, dt)
+    t = synth.codec_inputs(wl, seed=1)
+    codec = Codec(dt, to_device(t["U"], dt))
+    X = to_device(t["X"], dt)
+    Z = torch.empty((wl.n_tokens, 8), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(binding.SsnError) as e:
+        binding.ssn_compress_sum(codec.c, X.data_ptr(), 128, 0, 128, 0, 0, wl.n_tokens, 64, Z.data_ptr(), 8)
+    assert e.value.status == binding.SSN_ERR_NULL
+    with pytest.raises(binding.SsnError) as e:
+        binding.ssn_compress_sum(codec.c, X.data_ptr(), 128, X.data_ptr(), 64, 0, 0, wl.n_tokens, 64, Z.data_ptr(), 8)
+    assert e.value.status == binding.SSN_ERR_SHAPE
+    with pytest.raises(binding.SsnError) as e:
+        binding.ssn_compress_sum(codec.c, X.data_ptr(), 128, X.data_ptr(), 128, 0, 0, wl.n_tokens, 64, Z.data_ptr(), 8, 7)
+    assert e.value.status == binding.SSN_ERR_DTYPE

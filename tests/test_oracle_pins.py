@@ -444,3 +444,30 @@ def test_wire_round_trip_half_ulp():
     # values that are float32 already travel unchanged
     Z32 = Z.astype(np.float32).astype(np.float64)
     assert np.array_equal(oracle.wire_unpack(oracle.wire_rows(Z32), 11, False)[0], Z32)
+
+
+# ---- compress fused with the residual add ------------------------------------------------------
+def test_compress_sum_linearity_and_recovery():
+    rng = np.random.default_rng(11)
+    n, d, k, V, S = 9, 12, 4, 7, 5
+    U, _ = np.linalg.qr(rng.standard_normal((d, k)))
+    E, P = rng.standard_normal((V, d)), rng.standard_normal((S, d))
+    ids, pos = rng.integers(0, V, n), np.arange(n) % S
+    X, R = rng.standard_normal((n, d)), rng.standard_normal((n, d))
+    Zs, status = oracle.compress_sum(X, R, U, E, ids, P, pos)
+    assert status == 0
+    RU = np.zeros((n, k))                                  # R U with loops
+    for t_ in range(n):
+        for j in range(k):
+            for i in range(d):
+                RU[t_, j] += R[t_, i] * U[i, j]
+    np.testing.assert_allclose(Zs - oracle.compress(X, U, E, ids, P, pos)[0], RU, atol=1e-12)
+    # a hidden state split in two parts inside the shifted subspace gives the summed coordinates back
+    Za, Zb = rng.standard_normal((n, k)), rng.standard_normal((n, k))
+    Xa = Za @ U.T + E[ids] + P[pos]
+    Rb = Zb @ U.T
+    np.testing.assert_allclose(oracle.compress_sum(Xa, Rb, U, E, ids, P, pos)[0], Za + Zb, atol=1e-12)
+    # swapping the addends changes nothing; a zero residual is plain compress
+    np.testing.assert_allclose(oracle.compress_sum(R, X, U, E, ids, P, pos)[0], Zs, atol=1e-12)
+    np.testing.assert_array_equal(oracle.compress_sum(X, np.zeros_like(X), U, E, ids, P, pos)[0],
+                                  oracle.compress(X, U, E, ids, P, pos)[0])
