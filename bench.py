@@ -61,7 +61,7 @@ def parse_args():
                          "the E and P rows (the default step gathers; the table variant is always "
                          "timed beside it as compress_prepared_tables)")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
-    ap.add_argument("--sweep", choices=["compress", "reproject", "reparam", "wire"], default=None,
+    ap.add_argument("--sweep", choices=["compress", "reproject", "reparam", "wire", "dp"], default=None,
                     help="instead of the step: time the compress sweep (d, k, tokens) or the "
                          "re-projection sweep (k, weight shape, 32 layers); one JSON line per point")
     return ap.parse_args()
@@ -485,6 +485,58 @@ def run_sweep(args):
         print(json.dumps({"sweep": "reparam", "op": "head_embed", "tokens": n, "d": d, "k": k,
                           "us": round(us, 1), "GBps": round(algo / us / 1e3, 0),
                           "frac_of_measured": round(algo / us / 1e3 / peak, 3)}), flush=True)
+    elif args.sweep == "dp":
+        # AsyncSPARTA round steps and stage-wise clipping on one body stage of the 8B model:
+        # 8.03e9 / 7 parameters in fp32, the 5 % segment of a round (229 MB, larger than L2), 4 senders
+        from paper_2607_13332_b200 import dp_ops
+        n_params = 8_030_261_248 // 7
+        lo, hi = dp_ops.sparta_segment(n_params, 20, 7)
+        seg = hi - lo
+        theta = torch.randn(n_params, device="cuda", generator=gen)
+        senders = 4
+        chunks = [torch.randn(seg, device="cuda", generator=gen) for _ in range(senders)]
+        outs = [torch.empty(seg, device="cuda") for _ in range(senders)]
+        acc = torch.zeros(seg, device="cuda")
+        snap = torch.empty(seg, device="cuda")
+        ptr = lambda x: x.data_ptr()
+        points = [
+            ("sparta_snapshot", lambda: binding.sparta_snapshot(ptr(theta), lo, hi, ptr(snap)), 2 * seg * 4),
+            ("sparta_accumulate", lambda: binding.sparta_accumulate(ptr(acc), ptr(chunks[0]), 0.25, seg), 3 * seg * 4),
+            ("sparta_deltas, 4 senders",
+             lambda: binding.sparta_deltas(ptr(acc), 1.0, [ptr(c) for c in chunks], [ptr(o) for o in outs], seg),
+             (2 + 2 * senders) * seg * 4),
+            ("sparta_add_delta", lambda: binding.sparta_add_delta(ptr(theta), lo, hi, ptr(outs[0])), 3 * seg * 4),
+            ("sparta_apply_round", lambda: binding.sparta_apply_round(ptr(theta), lo, hi, ptr(acc), ptr(snap), 1.0),
+             4 * seg * 4),
+        ]
+        mib = (2 << 20) // 4                                  # one 2 MiB chunk of the round's stream
+        points.append(("sparta_accumulate, one 2 MiB chunk (L2-resident, launch-bound)",
+                       lambda: binding.sparta_accumulate(ptr(acc), ptr(chunks[0]), 0.25, mib), 3 * mib * 4))
+        for name, fn, algo in points:
+            us = timed_us(fn, 10)
+            print(json.dumps({"sweep": "dp", "op": name, "elements": seg if "MiB" not in name else mib,
+                              "us": round(us, 1), "GBps": round(algo / us / 1e3, 0),
+                              "frac_of_measured": round(algo / us / 1e3 / peak, 3)}), flush=True)
+        del chunks, outs, acc, snap
+        sumsq = torch.zeros(1, dtype=torch.float64, device="cuda")
+        thr = binding.stage_clip_threshold(7, False)
+        for tdt, code, size in ((torch.float32, binding.SSN_F32, 4), (torch.bfloat16, binding.SSN_BF16, 2)):
+            grad = (theta * 1e-3).to(tdt)
+            for name, fn, algo in (
+                    ("stage_clip_sumsq", lambda: binding.stage_clip_sumsq(ptr(grad), n_params, code, ptr(sumsq)),
+                     n_params * size),
+                    ("stage_clip_scale (outside the budget: read and write)",
+                     lambda: binding.stage_clip_scale(ptr(grad), n_params, code, ptr(sumsq), 1e-30),
+                     2 * n_params * size),
+                    ("stage_clip_scale (inside the budget: nothing to do)",
+                     lambda: binding.stage_clip_scale(ptr(grad), n_params, code, ptr(sumsq), 1e30), 0)):
+                sumsq.zero_()
+                binding.stage_clip_sumsq(ptr(grad), n_params, code, ptr(sumsq))
+                us = timed_us(fn, 5)
+                print(json.dumps({"sweep": "dp", "op": name, "dtype": "f32" if size == 4 else "bf16",
+                                  "elements": n_params, "us": round(us, 1), "GBps": round(algo / us / 1e3, 0),
+                                  "frac_of_measured": round(algo / us / 1e3 / peak, 3)}), flush=True)
+            del grad
     elif args.sweep == "wire":
         # wire rows (k fp32 coordinates + the token id) at the benchmark's stage boundary, next to the
         # storage-dtype calls of the step; ranks 24 and 40: decompress with one / two coordinate groups

@@ -79,6 +79,15 @@ _SIGNATURES = {
     "ssn_weight_reproject_list": (_i32, [_codec_p, ctypes.POINTER(_vp), ctypes.POINTER(_i64),
                                          ctypes.POINTER(_i64), _i32, _i32, _vp, _sz, _vp]),
     "ssn_static_scratch_bytes": (_sz, []),
+    "sparta_segment": (_i32, [_i64, _i32, _i64, ctypes.POINTER(_i64), ctypes.POINTER(_i64)]),
+    "sparta_snapshot": (_i32, [_vp, _i64, _i64, _vp, _vp]),
+    "sparta_accumulate": (_i32, [_vp, _vp, ctypes.c_float, _i64, _vp]),
+    "sparta_deltas": (_i32, [_vp, ctypes.c_float, ctypes.POINTER(_vp), ctypes.POINTER(_vp), _i32, _i64, _vp]),
+    "sparta_add_delta": (_i32, [_vp, _i64, _i64, _vp, _vp]),
+    "sparta_apply_round": (_i32, [_vp, _i64, _i64, _vp, _vp, ctypes.c_float, _vp]),
+    "stage_clip_threshold": (ctypes.c_float, [_i32, _i32]),
+    "stage_clip_sumsq": (_i32, [_vp, _i64, _i32, _vp, _vp]),
+    "stage_clip_scale": (_i32, [_vp, _i64, _i32, _vp, ctypes.c_float, _vp]),
     "ssn_status_string": (ctypes.c_char_p, [_i32]),
     "ssn_version": (_i32, []),
     "ssn_launch_count": (_i64, []),
@@ -96,7 +105,7 @@ def declared_symbols(header_dir: Optional[str] = None):
         if fname.endswith(".h"):
             text = open(os.path.join(header_dir, fname)).read()
             text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-            names += re.findall(r"\b(ssn_[a-z0-9_]+)\s*\(", text)
+            names += re.findall(r"\b((?:ssn|sparta|stage_clip)_[a-z0-9_]+)\s*\(", text)
     return sorted(set(names))
 
 
@@ -258,3 +267,47 @@ def ssn_prepare_tables(codec: ssn_codec_t, EU: int, ldeu: int, PU: int, ldpu: in
 def raw(name: str):
     """The raw ctypes function (returns the status instead of raising); used by error tests."""
     return getattr(_lib, name)
+
+
+# ---- data-parallel device ops (include/agora_dp.h) --------------------------------------------
+def sparta_segment(n_params: int, rounds_per_cycle: int, rnd: int):
+    lo, hi = _i64(0), _i64(0)
+    _check(_lib.sparta_segment(n_params, rounds_per_cycle, rnd, ctypes.byref(lo), ctypes.byref(hi)), "sparta_segment")
+    return int(lo.value), int(hi.value)
+
+
+def sparta_snapshot(buf: int, lo: int, hi: int, snap: int, stream: int = 0) -> None:
+    _check(_lib.sparta_snapshot(buf or None, lo, hi, snap or None, stream or None), "sparta_snapshot")
+
+
+def sparta_accumulate(acc: int, chunk: int, w: float, count: int, stream: int = 0) -> None:
+    _check(_lib.sparta_accumulate(acc or None, chunk or None, w, count, stream or None), "sparta_accumulate")
+
+
+def sparta_deltas(acc: int, sum_w: float, chunks, deltas, count: int, stream: int = 0) -> None:
+    n = len(chunks)
+    c_arr = (_vp * max(n, 1))(*chunks)
+    d_arr = (_vp * max(n, 1))(*deltas)
+    _check(_lib.sparta_deltas(acc or None, sum_w, c_arr, d_arr, n, count, stream or None), "sparta_deltas")
+
+
+def sparta_add_delta(buf: int, lo: int, hi: int, delta: int, stream: int = 0) -> None:
+    _check(_lib.sparta_add_delta(buf or None, lo, hi, delta or None, stream or None), "sparta_add_delta")
+
+
+def sparta_apply_round(theta: int, lo: int, hi: int, avg: int, snap: int, lam: float = 1.0, stream: int = 0) -> None:
+    _check(_lib.sparta_apply_round(theta or None, lo, hi, avg or None, snap or None, lam, stream or None),
+           "sparta_apply_round")
+
+
+def stage_clip_threshold(n_stages: int, is_tail: bool) -> float:
+    return float(_lib.stage_clip_threshold(n_stages, 1 if is_tail else 0))
+
+
+def stage_clip_sumsq(grad: int, count: int, dtype: int, sumsq: int, stream: int = 0) -> None:
+    _check(_lib.stage_clip_sumsq(grad or None, count, dtype, sumsq or None, stream or None), "stage_clip_sumsq")
+
+
+def stage_clip_scale(grad: int, count: int, dtype: int, sumsq: int, threshold: float, stream: int = 0) -> None:
+    _check(_lib.stage_clip_scale(grad or None, count, dtype, sumsq or None, threshold, stream or None),
+           "stage_clip_scale")

@@ -471,3 +471,90 @@ def test_compress_sum_linearity_and_recovery():
     np.testing.assert_allclose(oracle.compress_sum(R, X, U, E, ids, P, pos)[0], Zs, atol=1e-12)
     np.testing.assert_array_equal(oracle.compress_sum(X, np.zeros_like(X), U, E, ids, P, pos)[0],
                                   oracle.compress(X, U, E, ids, P, pos)[0])
+
+
+# ---- data-parallel ops: AsyncSPARTA round, stage-wise clipping ---------------------------------
+def test_sparta_round_from_steps_is_the_plain_mean():
+    """Eq. sparta: after a round every replica's buf[I] is the mean over replicas; assembled here
+    from the steps of Algorithm 3 with equal weights, and a weighted round with a weight-0 sender."""
+    from oracle import dp_oracle as dp
+    rng = np.random.default_rng(2)
+    n, R = 2003, 4
+    bufs = [rng.standard_normal(n) for _ in range(R)]
+    lo, hi = dp.sparta_segment(n, 20, 7)
+    assert (lo, hi) == (640, 768)                            # floor(701.05) and floor(801.2) down to 64s
+    for weights in ([1.0] * R, [3.0, 0.0, 1.0, 2.0]):
+        chunks = [dp.sparta_snapshot(b, lo, hi) for b in bufs]
+        acc = np.zeros(hi - lo)
+        for c, w in zip(chunks, weights):
+            acc = dp.sparta_accumulate(acc, c, w)
+        mean, deltas = dp.sparta_deltas(acc, sum(weights), chunks)
+        expect = sum(w * b[lo:hi] for w, b in zip(weights, bufs)) / sum(weights)
+        np.testing.assert_allclose(mean, expect, atol=1e-13)
+        for b, dlt in zip(bufs, deltas):
+            after = dp.sparta_add_delta(b, lo, hi, dlt)
+            np.testing.assert_allclose(after[lo:hi], expect, atol=1e-13)      # the group average
+            assert np.array_equal(after[:lo], b[:lo]) and np.array_equal(after[hi:], b[hi:])
+    # the weight-0 sender (index 1) changed nothing for the others: same mean without it
+    rest = [0, 2, 3]
+    np.testing.assert_allclose(expect, sum([3.0, 1.0, 2.0][i] * bufs[j][lo:hi] for i, j in enumerate(rest)) / 6.0,
+                               atol=1e-13)
+
+
+def test_sparta_segments_tile_a_cycle():
+    from oracle import dp_oracle as dp
+    for n in (0, 1, 19, 20, 1000, 8_030_261_248 // 7):
+        covered = 0
+        for r in range(20):
+            lo, hi = dp.sparta_segment(n, 20, r)
+            assert lo == covered and hi >= lo and lo % 64 == 0
+            assert abs(lo - n * r / 20) < 64                 # within one alignment unit of the even split
+            covered = hi
+        assert covered == n
+        assert dp.sparta_segment(n, 20, 27) == dp.sparta_segment(n, 20, 7)
+
+
+def test_delta_rule_keeps_local_progress():
+    """Eq. delta_rule: theta + (avg - snap); the local update theta - snap survives on top of the
+    average, and with no local progress (theta == snap) the result is the average itself."""
+    from oracle import dp_oracle as dp
+    rng = np.random.default_rng(3)
+    n, lo, hi = 50, 10, 30
+    theta, snap_full = rng.standard_normal(n), rng.standard_normal(n)
+    avg = rng.standard_normal(hi - lo)
+    snap = snap_full[lo:hi]
+    out = dp.sparta_apply_round(theta, lo, hi, avg, snap)
+    np.testing.assert_allclose(out[lo:hi] - avg, theta[lo:hi] - snap, atol=1e-13)
+    assert np.array_equal(out[:lo], theta[:lo]) and np.array_equal(out[hi:], theta[hi:])
+    np.testing.assert_allclose(dp.sparta_apply_round(snap_full, lo, hi, avg, snap)[lo:hi], avg, atol=1e-13)
+    np.testing.assert_allclose(dp.sparta_apply_round(theta, lo, hi, avg, snap, lam=0.0), theta, atol=0)
+
+
+def test_stage_clip_thresholds_printed_in_the_paper():
+    """Table 1 lists 0.3779 / 0.3779 / 0.7558 for head / body / tail of the 7-stage run."""
+    from oracle import dp_oracle as dp
+    golden = [float(v) for v in open(os.path.join(os.path.dirname(__file__), "golden",
+                                                  "stage_clip_thresholds.txt")).read().split()[-3:]]
+    assert golden == [0.3779, 0.3779, 0.7558]
+    assert abs(dp.stage_clip_threshold(7, False) - golden[0]) < 1e-4
+    assert abs(dp.stage_clip_threshold(7, True) - golden[2]) < 2e-4
+    assert dp.stage_clip_threshold(1, False) == 1.0          # one stage: the usual global threshold of 1
+    # S stages at their thresholds stay inside the unit budget: sum of squares = 1
+    assert abs(sum(dp.stage_clip_threshold(7, False) ** 2 for _ in range(7)) - 1.0) < 1e-12
+
+
+def test_stage_clip_norm_and_identity():
+    from oracle import dp_oracle as dp
+    rng = np.random.default_rng(4)
+    grads = [rng.standard_normal((5, 7)), rng.standard_normal(11), rng.standard_normal((2, 3, 4))]
+    norm = np.sqrt(sum(float((g ** 2).sum()) for g in grads))
+    c = 0.3779
+    clipped, got_norm, coef = dp.stage_clip(grads, c)
+    assert abs(got_norm - norm) < 1e-12 and coef < 1
+    new_norm = np.sqrt(sum(float((g ** 2).sum()) for g in clipped))
+    assert abs(new_norm - c) < 1e-5                          # min(norm, c) up to the 1e-6 guard
+    for g, h in zip(grads, clipped):                         # the direction is unchanged
+        np.testing.assert_allclose(h * norm, g * new_norm, atol=1e-12)
+    small = [g * (0.1 / norm) for g in grads]
+    same, _, coef1 = dp.stage_clip(small, c)
+    assert coef1 == 1.0 and all(np.array_equal(a, b) for a, b in zip(same, small))
