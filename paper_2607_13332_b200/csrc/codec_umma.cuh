@@ -514,12 +514,25 @@ codec_umma_project_kernel(const MmaArgs a, const __grid_constant__ UmmaMaps maps
       if (t < a.n) {
         // terms that come from the prepared tables E U and P U (fp32) instead of an operand
         auto subtract_row = [&](const float *row) {
+          const bool vec4 = (reinterpret_cast<uintptr_t>(row) & 15) == 0;   // 128-bit loads inside the row
 #pragma unroll
           for (int q = 0; q < Cfg::kN / 16; ++q)
 #pragma unroll
-            for (int i = 0; i < 16; ++i)
-              if (q * 16 + i < a.k)
-                v[q][i] = __float_as_uint(__uint_as_float(v[q][i]) - __ldg(row + q * 16 + i));
+            for (int i = 0; i < 16; i += 4) {
+              const int col = q * 16 + i;
+              if (vec4 && col + 4 <= a.k) {
+                const float4 w = __ldg(reinterpret_cast<const float4 *>(row + col));
+                v[q][i] = __float_as_uint(__uint_as_float(v[q][i]) - w.x);
+                v[q][i + 1] = __float_as_uint(__uint_as_float(v[q][i + 1]) - w.y);
+                v[q][i + 2] = __float_as_uint(__uint_as_float(v[q][i + 2]) - w.z);
+                v[q][i + 3] = __float_as_uint(__uint_as_float(v[q][i + 3]) - w.w);
+              } else {
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+                  if (col + e < a.k)
+                    v[q][i + e] = __float_as_uint(__uint_as_float(v[q][i + e]) - __ldg(row + col + e));
+              }
+            }
         };
         if (!HAS_E && a.shift.EU != nullptr) {
           const int64_t er = embedding_row(a.shift, t);

@@ -386,12 +386,20 @@ codec_umma_expand_kernel(const MmaArgs a, const ExpandGeometry geo, const __grid
             if (rows_live) tma_store_3d(&maps.out, slab, q * kChunkCols + g * 64, s1, s2);
             bulk_commit();
             if (HAS_E) {
-              // the store before this one is done reading its stage: hand that stage back
-              bulk_wait_read<1>();
-              if (held >= 0) mbar_arrive(e_empty_bar(held));
+              // the store before this one is done reading its stage: hand that stage back; after
+              // the chunk's last store wait for that one too, since this warp's next store is
+              // two chunks away and the stage would sit idle until then
+              if (g == kChunkCols / 64 - 1) {
+                bulk_wait_read<0>();
+                if (held >= 0) mbar_arrive(e_empty_bar(held));
+                mbar_arrive(e_empty_bar(eslot));
+              } else {
+                bulk_wait_read<1>();
+                if (held >= 0) mbar_arrive(e_empty_bar(held));
+              }
             }
           }
-          held = eslot;
+          held = g == kChunkCols / 64 - 1 ? -1 : eslot;
         }
       }
     }
