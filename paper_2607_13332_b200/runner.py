@@ -75,15 +75,17 @@ class Codec:
             P.data_ptr() if P is not None else 0, _ld(P) if P is not None else None,
             P.shape[0] if P is not None else 0)
 
-    def prepare_tables(self) -> None:
+    def prepare_tables(self, embedding: bool = True, positions: bool = True) -> None:
         """Project the codec's constant tables once (EU = E U, PU = P U, fp32) and attach them,
-        so that compress reads 2k floats per token instead of the E and P rows.  Call it again
-        after changing U, E or P in place."""
+        so that compress reads k floats per token and table instead of the E and P rows.  Either
+        table alone is allowed: PU is only seq_len x k and takes microseconds to make.  Call it
+        again after changing U, E or P in place."""
         dev = self.U.device
-        self.EU = torch.empty((self.E.shape[0], self.k), dtype=torch.float32, device=dev) \
-            if self.E is not None else None
-        self.PU = torch.empty((self.P.shape[0], self.k), dtype=torch.float32, device=dev) \
-            if self.P is not None else None
+        self.drop_tables()
+        if embedding and self.E is not None:
+            self.EU = torch.empty((self.E.shape[0], self.k), dtype=torch.float32, device=dev)
+        if positions and self.P is not None:
+            self.PU = torch.empty((self.P.shape[0], self.k), dtype=torch.float32, device=dev)
         binding.ssn_prepare_tables(self.c, self.EU.data_ptr() if self.EU is not None else 0, self.k,
                                    self.PU.data_ptr() if self.PU is not None else 0, self.k, _stream())
         if self.EU is not None:
