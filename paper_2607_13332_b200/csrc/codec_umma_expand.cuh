@@ -49,6 +49,10 @@ template <int KG, bool HAS_E, bool HAS_P>
 struct UmmaExpandConfig {
   static constexpr int kTileBytes = kUmmaTile * 128;            // [128 rows x 128 B]
   static constexpr int kZBytes = KG * kTileBytes;               // one Z tile: KG groups of 64 coordinates
+  // With E and two coordinate groups the E ring would have 4 stages only: one Z tile instead of two
+  // buys two more (the MMAs run up to two chunks ahead of the epilogue, which hides most of the
+  // load of the next tile's Z).  With one group the ring is deep enough and the second tile pays.
+  static constexpr int kZBufs = (HAS_E && KG == 2) ? 1 : 2;
   static constexpr int kU2Bytes = KG * kChunkCols * 128;        // 128 rows of U, K-major, KG groups
   static constexpr int kPBytes = HAS_P ? 2 * kGridPos * 128 : 0;   // 16 rows of P, two 64-column groups
   static constexpr int kUStageBytes = kU2Bytes + kPBytes;
@@ -58,10 +62,10 @@ struct UmmaExpandConfig {
   // sum is formed in place in the E stage, which is then the source of the TMA store.
   static constexpr int kStagingBytes = HAS_E ? 0 : 8 * 2 * 4096;
   static constexpr int kFixedBytes =
-      2 * kZBytes + (HAS_P ? kTileBytes : 0) + kUStages * kUStageBytes + kStagingBytes;
+      kZBufs * kZBytes + (HAS_P ? kTileBytes : 0) + kUStages * kUStageBytes + kStagingBytes;
   static constexpr int kMaxSmem = 227 * 1024;
   static constexpr int kEFit = (kMaxSmem - 1024 - 512 - kFixedBytes) / kEStageBytes;
-  static constexpr int kEStages = HAS_E ? (kEFit < 8 ? kEFit : 8) : 0;
+  static constexpr int kEStages = HAS_E ? (kEFit < 12 ? kEFit : 12) : 0;
   static_assert(!HAS_E || kEStages >= 4, "no room for the E ring");
   static constexpr int kTmemCols = 256;
   static constexpr int SE = HAS_E ? kEStages : 1;
@@ -94,8 +98,8 @@ codec_umma_expand_kernel(const MmaArgs a, const ExpandGeometry geo, const __grid
   const int64_t ntiles = geo.ntiles;
 
   const uint32_t smem0 = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  const uint32_t z_base = smem0;                                         // two Z tiles
-  const uint32_t sel = z_base + 2 * Cfg::kZBytes;                        // selection matrix (HAS_P)
+  const uint32_t z_base = smem0;                                         // the Z tiles
+  const uint32_t sel = z_base + Cfg::kZBufs * Cfg::kZBytes;              // selection matrix (HAS_P)
   const uint32_t u_ring = sel + (HAS_P ? Cfg::kTileBytes : 0);
   const uint32_t staging = u_ring + SU * Cfg::kUStageBytes;
   const uint32_t e_ring = staging + Cfg::kStagingBytes;
@@ -190,8 +194,8 @@ codec_umma_expand_kernel(const MmaArgs a, const ExpandGeometry geo, const __grid
     for (int64_t tile = tile_lo; tile <= tile_hi; ++tile, ++tcount) {
       int c1, c2;
       tile_coords(tile, c1, c2);
-      const int zb = (int)(tcount & 1);
-      if (!dead && !mbar_wait(z_empty_bar(zb), (uint32_t)(((tcount >> 1) & 1) ^ 1))) timed_out();
+      const int zb = (int)(tcount % Cfg::kZBufs);
+      if (!dead && !mbar_wait(z_empty_bar(zb), (uint32_t)(((tcount / Cfg::kZBufs) & 1) ^ 1))) timed_out();
       if (lane == 0) {
         mbar_expect_tx(z_full_bar(zb), Cfg::kZBytes);
 #pragma unroll
@@ -235,8 +239,8 @@ codec_umma_expand_kernel(const MmaArgs a, const ExpandGeometry geo, const __grid
       uint32_t parity = 0;
       int64_t tcount = 0, ccount = 0;
       for (int64_t tile = tile_lo; tile <= tile_hi; ++tile, ++tcount) {
-        const int zb = (int)(tcount & 1);
-        if (!dead && !mbar_wait(z_full_bar(zb), (uint32_t)((tcount >> 1) & 1))) timed_out();
+        const int zb = (int)(tcount % Cfg::kZBufs);
+        if (!dead && !mbar_wait(z_full_bar(zb), (uint32_t)((tcount / Cfg::kZBufs) & 1))) timed_out();
         const uint64_t zd = kdesc + umma_desc_addr(z_base + zb * Cfg::kZBytes);
         int q0, q1;
         chunk_range(tile, q0, q1);
