@@ -8,6 +8,7 @@
 #include "codec_umma_tokens.cuh"
 
 
+#include <cstdlib>
 #include "codec_mma_launch.h"
 
 namespace ssn {
@@ -400,7 +401,9 @@ cudaError_t launch_codec_umma_expand(const MmaArgs &a, bool shift, int sm_count,
       return cudaErrorNotSupported;
     if (!make_sw128_map3(&maps.out, a.dst, a.d, L, B, a.lddst, L * a.lddst, kGridPos, 32 / kGridPos))
       return cudaErrorNotSupported;
-    if (!make_sw128_map(&maps.p, a.shift.P, a.shift.max_pos, a.d, a.shift.ldp, kGridPos))
+    // P as [column group of 64][position][64 columns]: one box of 64 x 16 x 2 is a chunk's 16 rows
+    if (!make_sw128_map3(&maps.p, a.shift.P, kUmmaCols, a.shift.max_pos, a.d / kUmmaCols, a.shift.ldp, kUmmaCols,
+                         kGridPos, kChunkCols / kUmmaCols))
       return cudaErrorNotSupported;
   } else {
     if (!make_sw128_map3(&maps.z, a.zin, a.k, a.n, 1, a.ldzin, a.n * a.ldzin, kUmmaTile, 1))

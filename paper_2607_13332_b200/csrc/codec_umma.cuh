@@ -81,6 +81,24 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map
       "cp.async.bulk.tensor.2d.shared::cta.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];\n"
       ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1) : "memory");
 }
+// L2 eviction policies for the copies below: evict_first for what streams through once (so that
+// it does not push out what comes back), evict_last for the small operands every tile re-reads.
+__device__ __forceinline__ uint64_t l2_policy_evict_last() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;\n" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;\n" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ void tma_load_2d_hint(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1,
+                                                 uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cta.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4}], [%2], %5;\n"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "l"(policy) : "memory");
+}
 __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *map, uint32_t bar,
                                             int c0, int c1, int c2, int c3) {
   asm volatile(
@@ -287,6 +305,8 @@ codec_umma_project_kernel(const MmaArgs a, const __grid_constant__ UmmaMaps maps
 
   if (warp == 0) {
     // ------------------------------------------------------------------------- producer
+    // the rows to project pass through L2 once; the P rows come back for every sequence
+    const uint64_t stream_in = l2_policy_evict_first(), keep = l2_policy_evict_last();
     int slot = 0;
     uint32_t parity = 1;   // a fresh "empty" barrier passes a wait on parity 1
     int64_t cached_blk = -1;
@@ -305,8 +325,8 @@ codec_umma_project_kernel(const MmaArgs a, const __grid_constant__ UmmaMaps maps
         if (lane == 0) {
           mbar_expect_tx(bar, Cfg::kTmaBytes - (HAS_P && !load_p ? Cfg::kATileBytes : 0));
           const int su = st < nstage1 ? st : st - nstage1;   // slice of U; the second matrix starts over
-          tma_load_2d(base, st < nstage1 ? &maps.x : &maps.x2, bar, su * kUmmaCols, (int)tok0);
-          if (load_p) tma_load_2d(base + kPTile * Cfg::kATileBytes, &maps.p, bar, st * kUmmaCols, pos0);
+          tma_load_2d_hint(base, st < nstage1 ? &maps.x : &maps.x2, bar, su * kUmmaCols, (int)tok0, stream_in);
+          if (load_p) tma_load_2d_hint(base + kPTile * Cfg::kATileBytes, &maps.p, bar, st * kUmmaCols, pos0, keep);
 #pragma unroll
           for (int ug = 0; ug < Cfg::kUGroups; ++ug)
             tma_load_2d(base + Cfg::kATiles * Cfg::kATileBytes + ug * Cfg::kUGroupBytes,

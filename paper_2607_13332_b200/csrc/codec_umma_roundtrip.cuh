@@ -40,6 +40,10 @@ __device__ __forceinline__ void tma_store_2d(const CUtensorMap *map, uint32_t sr
   asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];\n"
                ::"l"(map), "r"(src), "r"(c0), "r"(c1) : "memory");
 }
+__device__ __forceinline__ void tma_store_2d_hint(const CUtensorMap *map, uint32_t src, int c0, int c1, uint64_t policy) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group.L2::cache_hint [%0, {%2, %3}], [%1], %4;\n"
+               ::"l"(map), "r"(src), "r"(c0), "r"(c1), "l"(policy) : "memory");
+}
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;\n" ::: "memory"); }
 template <int N> __device__ __forceinline__ void bulk_wait_read() {
   asm volatile("cp.async.bulk.wait_group.read %0;\n" ::"n"(N) : "memory");
@@ -166,6 +170,7 @@ codec_umma_roundtrip_kernel(const MmaArgs a, const __grid_constant__ UmmaRoundTr
 
   if (warp == 0) {
     // ------------------------------------------------------------------------- pass-1 producer
+    const uint64_t stream_in = l2_policy_evict_first();   // every tile is read once
     int slot = 0;
     uint32_t parity = 1;   // a fresh "empty" barrier passes a wait on parity 1
     for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
@@ -177,10 +182,10 @@ codec_umma_roundtrip_kernel(const MmaArgs a, const __grid_constant__ UmmaRoundTr
         if (lane == 0) {
           mbar_expect_tx(full_bar(slot), Cfg::kStageBytes);
           if (LEFT) {   // rows st*64.. of the column block: two boxes of 64 columns
-            tma_load_2d(base, &maps.s[w], full_bar(slot), row0, st * kUmmaCols);
-            tma_load_2d(base + Cfg::kTileBytes / 2, &maps.s[w], full_bar(slot), row0 + 64, st * kUmmaCols);
+            tma_load_2d_hint(base, &maps.s[w], full_bar(slot), row0, st * kUmmaCols, stream_in);
+            tma_load_2d_hint(base + Cfg::kTileBytes / 2, &maps.s[w], full_bar(slot), row0 + 64, st * kUmmaCols, stream_in);
           } else {
-            tma_load_2d(base, &maps.s[w], full_bar(slot), st * kUmmaCols, row0);
+            tma_load_2d_hint(base, &maps.s[w], full_bar(slot), st * kUmmaCols, row0, stream_in);
           }
 #pragma unroll
           for (int ug = 0; ug < Cfg::kKG; ++ug)
@@ -285,6 +290,7 @@ codec_umma_roundtrip_kernel(const MmaArgs a, const __grid_constant__ UmmaRoundTr
     const int r = quarter * 32 + lane;
     const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16);
     const uint32_t slab0 = staging + (uint32_t)quarter * 8192;
+    const uint64_t stream_out = l2_policy_evict_first();   // written once, not read again here
     const bool zvec = a.zout != nullptr && ((a.ldzout & 7) == 0) && ((reinterpret_cast<uintptr_t>(a.zout) & 15) == 0);
     int64_t tcount = 0, ccount = 0;
     for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x, ++tcount) {
@@ -375,9 +381,9 @@ codec_umma_roundtrip_kernel(const MmaArgs a, const __grid_constant__ UmmaRoundTr
           if (lane == 0) {
             if (LEFT) {   // rows q*128 + 32*quarter .. of W, columns of this block
               if (row0 + g * 64 < nrows)
-                tma_store_2d(&maps.out[w], slab, row0 + g * 64, q * kChunkCols + quarter * 32);
+                tma_store_2d_hint(&maps.out[w], slab, row0 + g * 64, q * kChunkCols + quarter * 32, stream_out);
             } else if (row0 + quarter * 32 < nrows) {
-              tma_store_2d(&maps.out[w], slab, q * kChunkCols + g * 64, (int)(row0 + quarter * 32));
+              tma_store_2d_hint(&maps.out[w], slab, q * kChunkCols + g * 64, (int)(row0 + quarter * 32), stream_out);
             }
             bulk_commit();
           }

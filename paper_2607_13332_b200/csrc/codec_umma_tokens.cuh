@@ -98,6 +98,7 @@ codec_umma_tokens_kernel(const TokensArgs a, const __grid_constant__ UmmaTokensM
 
   if (warp == 0) {
     // ------------------------------------------------------------------------- producer
+    const uint64_t stream_in = l2_policy_evict_first();   // H is read once; C comes back for every column block
     int slot = 0;
     uint32_t parity = 1;
     for (int64_t st = st_lo; st < st_hi; ++st) {
@@ -106,8 +107,8 @@ codec_umma_tokens_kernel(const TokensArgs a, const __grid_constant__ UmmaTokensM
       if (lane == 0) {
         const int tok0 = (int)(st * kUmmaCols);
         mbar_expect_tx(full_bar(slot), Cfg::kStageBytes);
-        tma_load_2d(base, &maps.h, full_bar(slot), col0, tok0);
-        tma_load_2d(base + Cfg::kABytes / 2, &maps.h, full_bar(slot), col0 + 64, tok0);
+        tma_load_2d_hint(base, &maps.h, full_bar(slot), col0, tok0, stream_in);
+        tma_load_2d_hint(base + Cfg::kABytes / 2, &maps.h, full_bar(slot), col0 + 64, tok0, stream_in);
         // the last box of C would read past its buffer through the wide map
 #pragma unroll
         for (int g = 0; g < Cfg::kKG; ++g)
