@@ -40,9 +40,9 @@ FALLBACK_HBM_GBS = 6650.0
 
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of ONE launch of each kernel on the
 # default workload, from the ncu captures summarised under profiles/; None where not captured.
-NCU_TRAFFIC_BYTES = {"compress": None, "decompress": 705.7e6, "grad_project": 541.7e6,
-                     "weight_reproject": 238.7e6}
-NCU_TRAFFIC_COMPRESS = {True: 550.5e6, False: 729.5e6}     # keyed by "prepared tables"
+NCU_TRAFFIC_BYTES = {"compress": None, "decompress": 648.9e6, "grad_project": 540.2e6,
+                     "weight_reproject": 238.4e6}
+NCU_TRAFFIC_COMPRESS = {True: 550.5e6, False: 712.3e6}     # keyed by "prepared tables"
 
 
 REPROJECT_ROWS_COLS = ((4096, 4096), (14336, 4096))
