@@ -136,47 +136,44 @@ __global__ void gather_rows_kernel(const GatherArgs a) {
   static_cast<T *>(a.out)[t * a.ld_out + j] = v;
 }
 
-// ---- wire rows in: ids out of word k, coordinates as bf16 head + remainder -------------------
-struct WireSplitArgs {
+// ---- wire rows in: ids out of word k, coordinates as bf16 head + remainder; the basis twice -----
+// One launch prepares both operands of the split expansion.  Blocks are (kp x rows_per_block)
+// threads: thread (j, y) owns column j of one row, so nothing is divided.
+//   blocks [0, split_blocks):  row t of the wire buffer -> ids[t] (word k) and, when split is given,
+//       split[t] = (head | remainder) in columns [0, k) and [kp, kp + k), zeros elsewhere
+//   blocks [split_blocks, ..): row r of U -> U2[r] = (U[r] 0 | U[r] 0), so that
+//       (head | remainder) U2^T = (head + remainder) U^T
+struct WirePrepareArgs {
   const float *wire;        // [n x ldw] words
-  __nv_bfloat16 *split;     // [n x 2 kp] or nullptr: head in columns [0, k), remainder in [kp, kp + k), zeros elsewhere
-  int32_t *ids;             // [n] or nullptr: word k of every row
-  int64_t ldw, n;
-  int32_t k, kp;
+  __nv_bfloat16 *split;     // [n x 2 kp] or nullptr
+  int32_t *ids;             // [n] or nullptr
+  const __nv_bfloat16 *U;   // [d x k], leading dimension ldu (split only)
+  __nv_bfloat16 *U2;        // [d x 2 kp] (split only)
+  int64_t ldw, ldu, n;
+  int32_t k, kp, d;
+  int32_t split_blocks;
 };
 
-static __global__ void wire_split_kernel(const WireSplitArgs a) {
-  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  const int w = a.split != nullptr ? a.kp : 1;     // threads per row
-  if (i >= a.n * w) return;
-  const int64_t t = i / w;
-  const int j = (int)(i - t * w);
-  const float *row = a.wire + t * a.ldw;
-  if (a.ids != nullptr && j == 0) a.ids[t] = reinterpret_cast<const int32_t *>(row)[a.k];
-  if (a.split != nullptr) {
-    const float z = j < a.k ? row[j] : 0.f;
-    const __nv_bfloat16 head = __float2bfloat16_rn(z);
-    a.split[t * 2 * a.kp + j] = head;
-    a.split[t * 2 * a.kp + a.kp + j] = __float2bfloat16_rn(z - __bfloat162float(head));
+static __global__ void wire_prepare_kernel(const WirePrepareArgs a) {
+  const int j = threadIdx.x;
+  if ((int)blockIdx.x < a.split_blocks) {
+    const int64_t t = (int64_t)blockIdx.x * blockDim.y + threadIdx.y;
+    if (t >= a.n) return;
+    const float *row = a.wire + t * a.ldw;
+    if (a.ids != nullptr && j == 0) a.ids[t] = reinterpret_cast<const int32_t *>(row)[a.k];
+    if (a.split != nullptr) {
+      const float z = j < a.k ? row[j] : 0.f;
+      const __nv_bfloat16 head = __float2bfloat16_rn(z);
+      a.split[t * 2 * a.kp + j] = head;
+      a.split[t * 2 * a.kp + a.kp + j] = __float2bfloat16_rn(z - __bfloat162float(head));
+    }
+  } else {
+    const int64_t r = (int64_t)(blockIdx.x - a.split_blocks) * blockDim.y + threadIdx.y;
+    if (r >= a.d) return;
+    const __nv_bfloat16 v = j < a.k ? a.U[r * a.ldu + j] : __float2bfloat16_rn(0.f);
+    a.U2[r * 2 * a.kp + j] = v;
+    a.U2[r * 2 * a.kp + a.kp + j] = v;
   }
-}
-
-// U2 [d x 2 kp] = [U 0 | U 0]: the basis twice, so that (head | remainder) U2^T = (head + remainder) U^T
-struct BasisDupArgs {
-  const __nv_bfloat16 *U;
-  __nv_bfloat16 *U2;
-  int64_t ldu;
-  int32_t d, k, kp;
-};
-
-static __global__ void basis_dup_kernel(const BasisDupArgs a) {
-  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= (int64_t)a.d * a.kp) return;
-  const int64_t r = i / a.kp;
-  const int j = (int)(i - r * a.kp);
-  const __nv_bfloat16 v = j < a.k ? a.U[r * a.ldu + j] : __float2bfloat16_rn(0.f);
-  a.U2[r * 2 * a.kp + j] = v;
-  a.U2[r * 2 * a.kp + a.kp + j] = v;
 }
 
 // ---- contraction over tokens: out [m x k] (fp32) = H^T C, H [n x m], C [n x k] ---------------

@@ -558,21 +558,6 @@ ssn_status_t ssn_decompress_wire(const ssn_codec_t *codec, const void *wire, int
   const size_t split_bytes = round256((size_t)n_tokens * 2 * kp * 2), u2_bytes = round256((size_t)codec->d * 2 * kp * 2);
   const bool split = wire_split_fits(codec) && workspace != nullptr && (reinterpret_cast<uintptr_t>(workspace) & 255) == 0 &&
                      workspace_bytes >= ids_bytes + split_bytes + u2_bytes;
-  WireSplitArgs w{};
-  w.wire = static_cast<const float *>(wire);
-  w.ldw = ldw;
-  w.n = n_tokens;
-  w.k = codec->k;
-  w.kp = kp;
-  w.ids = ids_out;
-  w.split = split ? reinterpret_cast<__nv_bfloat16 *>(ws + ids_bytes) : nullptr;
-  if (w.ids != nullptr || w.split != nullptr) {
-    const int64_t threads = n_tokens * (split ? kp : 1), blocks = (threads + 255) / 256;
-    if (blocks > 0x7fffffffLL) return SSN_ERR_SHAPE;
-    wire_split_kernel<<<(unsigned)blocks, 256, 0, s>>>(w);
-    st = launch_status();
-    if (st != SSN_OK) return st;
-  }
   TokenArgs a{};
   st = make_shift(codec, with_ids ? ids_out : ids, pos, seq_len, dev_status, &a.shift);
   if (st != SSN_OK) return st;
@@ -581,24 +566,39 @@ ssn_status_t ssn_decompress_wire(const ssn_codec_t *codec, const void *wire, int
   a.n = n_tokens;
   a.d = codec->d;
   a.add_shift = 1;
-  if (split) {
-    BasisDupArgs b{};
-    b.U = static_cast<const __nv_bfloat16 *>(codec->U);
-    b.U2 = reinterpret_cast<__nv_bfloat16 *>(ws + ids_bytes + split_bytes);
-    b.ldu = codec->ldu;
-    b.d = codec->d;
-    b.k = codec->k;
-    b.kp = kp;
-    const int64_t blocks = ((int64_t)codec->d * kp + 255) / 256;
-    basis_dup_kernel<<<(unsigned)blocks, 256, 0, s>>>(b);
+  if (split || ids_out != nullptr) {
+    // one small launch: the ids out of the rows, and for the split form the two bf16 operands
+    WirePrepareArgs w{};
+    w.wire = static_cast<const float *>(wire);
+    w.ldw = ldw;
+    w.n = n_tokens;
+    w.k = codec->k;
+    w.kp = split ? kp : 1;
+    w.d = codec->d;
+    w.ids = ids_out;
+    const int rows_per_block = 256 / w.kp;
+    const int64_t split_blocks = (n_tokens + rows_per_block - 1) / rows_per_block;
+    const int64_t basis_blocks = split ? (codec->d + rows_per_block - 1) / rows_per_block : 0;
+    if (split_blocks + basis_blocks > 0x7fffffffLL) return SSN_ERR_SHAPE;
+    w.split_blocks = (int32_t)split_blocks;
+    if (split) {
+      w.split = reinterpret_cast<__nv_bfloat16 *>(ws + ids_bytes);
+      w.U = static_cast<const __nv_bfloat16 *>(codec->U);
+      w.ldu = codec->ldu;
+      w.U2 = reinterpret_cast<__nv_bfloat16 *>(ws + ids_bytes + split_bytes);
+    }
+    wire_prepare_kernel<<<(unsigned)(split_blocks + basis_blocks), dim3((unsigned)w.kp, (unsigned)rows_per_block), 0, s>>>(w);
     st = launch_status();
     if (st != SSN_OK) return st;
-    a.zin = w.split;
-    a.ldzin = 2 * kp;
-    a.U = b.U2;
-    a.ldu = 2 * kp;
-    a.k = 2 * kp;
-  } else {
+    if (split) {
+      a.zin = w.split;
+      a.ldzin = 2 * kp;
+      a.U = w.U2;
+      a.ldu = 2 * kp;
+      a.k = 2 * kp;
+    }
+  }
+  if (!split) {
     a.zin = wire;
     a.ldzin = ldw;
     a.wire = 1;
