@@ -22,7 +22,11 @@
 //              clips the rows past n).
 //   warps 10-13  gather the E rows of the tile, 64 columns at a time, with cp.async into
 //              swizzled stages (an id outside the table points at a row of zeros); the epilogue
-//              forms the sum in place and the stage is the source of the TMA store.
+//              forms the sum in place and the stage is the source of the TMA store; a stage
+//              goes back to the gather warps as soon as the chunk's last store has read it.
+// L2: the output is stored with an evict_first policy and the P rows are loaded with evict_last,
+// so that the streams do not push the 16 rows under a chunk out before the next group of
+// sequences needs them.
 // Every wait is bounded; a wait that runs out sets SSN_DEV_TIMEOUT and the kernel still ends.
 #pragma once
 
