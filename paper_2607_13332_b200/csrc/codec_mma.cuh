@@ -45,7 +45,7 @@ __device__ __forceinline__ void cp_async16(uint32_t dst, const void *src, int sr
 }
 // the same, not allocating in L1 (for rows that are read once)
 __device__ __forceinline__ void cp_async16_cg(uint32_t dst, const void *src) {
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(dst), "l"(src));
+  asm volatile("cp.async.cg.shared.global.L2::256B [%0], [%1], 16;\n" ::"r"(dst), "l"(src));
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::); }
 template <int N> __device__ __forceinline__ void cp_async_wait() {
