@@ -136,6 +136,19 @@ __global__ void gather_rows_kernel(const GatherArgs a) {
   static_cast<T *>(a.out)[t * a.ld_out + j] = v;
 }
 
+// The same with blocks of (kpad x rows) threads, thread (j, y) = column j of one row: no index
+// division (kpad <= 256).
+template <typename T>
+__global__ void gather_rows_2d_kernel(const GatherArgs a) {
+  const int64_t t = (int64_t)blockIdx.x * blockDim.y + threadIdx.y;
+  const int j = threadIdx.x;
+  if (t >= a.n) return;
+  const int64_t id = a.ids[t];
+  T v = from_f32<T>(0.f);
+  if (j < a.k && id >= 0 && id < a.rows) v = static_cast<const T *>(a.table)[id * a.ld_table + j];
+  static_cast<T *>(a.out)[t * a.ld_out + j] = v;
+}
+
 // ---- wire rows in: ids out of word k, coordinates as bf16 head + remainder; the basis twice -----
 // One launch prepares both operands of the split expansion.  Blocks are (kp x rows_per_block)
 // threads: thread (j, y) owns column j of one row, so nothing is divided.

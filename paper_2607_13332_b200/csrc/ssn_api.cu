@@ -736,13 +736,24 @@ ssn_status_t ssn_head_embed(const ssn_codec_t *codec, const void *Elow, int64_t 
   g.rows = vocab_low;
   g.k = codec->k;
   g.kpad = kpad;
-  const int64_t total = n_tokens * kpad, blocks = (total + 255) / 256;
-  if (blocks > 0x7fffffffLL) return SSN_ERR_SHAPE;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  if (codec->dtype == SSN_F32)
-    gather_rows_kernel<float><<<(unsigned)blocks, 256, 0, s>>>(g);
-  else
-    gather_rows_kernel<__nv_bfloat16><<<(unsigned)blocks, 256, 0, s>>>(g);
+  if (kpad <= 256) {
+    const int rows_per_block = 256 / (int)kpad;
+    const int64_t blocks = (n_tokens + rows_per_block - 1) / rows_per_block;
+    if (blocks > 0x7fffffffLL) return SSN_ERR_SHAPE;
+    const dim3 block((unsigned)kpad, (unsigned)rows_per_block);
+    if (codec->dtype == SSN_F32)
+      gather_rows_2d_kernel<float><<<(unsigned)blocks, block, 0, s>>>(g);
+    else
+      gather_rows_2d_kernel<__nv_bfloat16><<<(unsigned)blocks, block, 0, s>>>(g);
+  } else {
+    const int64_t total = n_tokens * kpad, blocks = (total + 255) / 256;
+    if (blocks > 0x7fffffffLL) return SSN_ERR_SHAPE;
+    if (codec->dtype == SSN_F32)
+      gather_rows_kernel<float><<<(unsigned)blocks, 256, 0, s>>>(g);
+    else
+      gather_rows_kernel<__nv_bfloat16><<<(unsigned)blocks, 256, 0, s>>>(g);
+  }
   st = launch_status();
   if (st != SSN_OK) return st;
   return ssn_decompress(codec, workspace, kpad, ids, pos, n_tokens, seq_len, X0, ldx, dev_status, stream);
