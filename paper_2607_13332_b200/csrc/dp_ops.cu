@@ -1,7 +1,7 @@
 // Data-parallel device ops (include/agora_dp.h): the elementwise steps of an AsyncSPARTA round
 // (Algorithm 3, Eq. sparta, Eq. delta_rule) and stage-wise gradient clipping (Sec. 4.3).  All of
 // them stream their operands once: grid-stride loops, 128-bit accesses when every pointer is
-// 16-byte aligned, a grid of a few blocks per SM.
+// 16-byte aligned, a grid of two waves of resident blocks.
 #include "agora_dp.h"
 
 #include <cuda_bf16.h>
@@ -13,7 +13,7 @@
 namespace {
 
 constexpr int kThreads = 256;
-constexpr int kBlocksPerSm = 8;
+constexpr int kBlocksPerSm = 16;
 
 inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 
