@@ -350,7 +350,7 @@ def run_ours(args):
     status = codec.take_status()
     status |= codec_t.take_status()
     if status != 0:
-        raise RuntimeError(f"device status {status}: synthetic ids/positions out of range")
+        raise RuntimeError(f"device status {status}: {Codec.describe_status(status)}")
 
     if rank == 0:
         ms_per_step = ms_total / args.steps

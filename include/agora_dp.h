@@ -4,7 +4,7 @@
  * and stage-wise gradient clipping (Sec. 4.3).  C ABI, raw DEVICE pointers unless a comment says
  * host, element counts, a cudaStream_t passed as void*; nothing is allocated, freed or
  * synchronised inside.  Parameter buffers are fp32, as the round's buffer is in Algorithm 3
- * ("refresh FP32 buf").  Status codes are those of ssn.h.  Buffers of one call must not overlap
+ * (its first step refreshes an fp32 copy).  Status codes are those of ssn.h.  Buffers of one call must not overlap
  * unless stated; 16-byte aligned pointers get 128-bit accesses, others element-wise ones.
  */
 #ifndef AGORA_DP_H_
@@ -17,7 +17,7 @@ extern "C" {
 #endif
 
 /*
- * The index set of a round (Algorithm 3: "fraction s of parameters, rotated by step", the same on
+ * The index set of a round (Algorithm 3: a fraction s of the parameters that rotates with the step, the same on
  * every peer; consecutive rounds cover every parameter once per 1/s rounds): the contiguous
  * segment [*lo, *hi) with r = round mod R, R = rounds_per_cycle (20 for s = 5 %),
  *     lo = floor(n r / R) rounded down to a multiple of SPARTA_SEGMENT_ALIGN,
@@ -29,11 +29,11 @@ extern "C" {
 ssn_status_t sparta_segment(int64_t n_params, int32_t rounds_per_cycle, int64_t round,
                             int64_t *lo, int64_t *hi);
 
-/* Algorithm 3, "snap <- copy(buf[P])": snap[0 : hi - lo] = buf[lo : hi]. */
+/* Algorithm 3, the snapshot step of a sender: snap[0 : hi - lo] = buf[lo : hi]. */
 ssn_status_t sparta_snapshot(const float *buf, int64_t lo, int64_t hi, float *snap, void *stream);
 
 /* Algorithm 3, reducer, per arriving chunk c_i of sender i: acc[0:count] += w * chunk[0:count]
- * (a sender with w = 0 "absorbs, adds nothing"). */
+ * (a sender of weight 0 takes part in the round without contributing). */
 ssn_status_t sparta_accumulate(float *acc, const float *chunk, float w, int64_t count, void *stream);
 
 /*
@@ -46,7 +46,7 @@ ssn_status_t sparta_accumulate(float *acc, const float *chunk, float w, int64_t 
 ssn_status_t sparta_deltas(float *acc, float sum_w, const float *const *chunks, float *const *deltas,
                            int32_t senders, int64_t count, void *stream);
 
-/* Algorithm 3, sender: "buf[P] += received deltas": buf[lo : hi] += delta[0 : hi - lo]. */
+/* Algorithm 3, sender, on receiving its deltas: buf[lo : hi] += delta[0 : hi - lo]. */
 ssn_status_t sparta_add_delta(float *buf, int64_t lo, int64_t hi, const float *delta, void *stream);
 
 /*

@@ -30,8 +30,17 @@
  *     position is outside [0, max_pos) takes a ZERO row for that term, and bit 0 (bad id) or
  *     bit 1 (bad position) is OR-ed into *dev_status when that pointer is not NULL.  The
  *     caller zeroes *dev_status beforehand.
+ *   - A tensor-core kernel's internal waits (on its own copies and accumulators) are bounded;
+ *     one that runs out ORs SSN_DEV_TIMEOUT into the status word and the kernel still ends.  The
+ *     output of that call is invalid then.  The status word is the call's dev_status argument
+ *     or, when that is NULL or the call has none, codec->dev_status.
  *   - Inputs and outputs of one call must not overlap, except ssn_weight_reproject, which
  *     works in place.
+ *   - Threads and devices: the library keeps no state a call's result depends on.  Its caches
+ *     (SM count, kernel attributes, the scratch address of the _static call) are per device,
+ *     filled on first use with atomic updates, so calls may come from several host threads and
+ *     for several devices (the current device of the calling thread is used, as for any
+ *     runtime call).  The diagnostics ssn_launch_count and ssn_last_kernel are informational.
  *   - bf16 buffers whose pointers are 16-byte aligned and whose leading dimensions are
  *     multiples of 8 take the vectorised tensor-core kernels; anything else (fp32, odd
  *     leading dimensions, unaligned views) is still computed, by slower general kernels.
@@ -71,8 +80,9 @@ typedef enum { SSN_GRAD_COEFF = 1, SSN_GRAD_FULL = 2 } ssn_grad_mode_t;
 #define SSN_DEV_TIMEOUT 4   /* an internal bounded wait ran out; the output is invalid */
 
 /*
- * The data both ends of a stage boundary share (Sec. 4.1: the basis U_k, and PE and T_fixed
- * "available to both sender and receiver").  Plain value struct; nothing is owned.
+ * The data both ends of a stage boundary share (Sec. 4.1, the paragraph before Eq.
+ * ssn_compress: the basis U_k, and the tables PE and T_fixed that sender and receiver both
+ * hold).  Plain value struct; nothing is owned.
  */
 /*
  * Performance note.  The tensor-core kernels need 16-byte aligned base addresses and leading
@@ -100,6 +110,9 @@ typedef struct ssn_codec {
   int64_t ldeu;         /* >= k                                                           */
   const float *PU;      /* device [max_pos x k] = P U, or NULL                            */
   int64_t ldpu;         /* >= k                                                           */
+  /* Optional device status word for the calls that take no dev_status argument (grad-project,
+   * re-projection, the reparameterized ops) and for the others when theirs is NULL.          */
+  int32_t *dev_status;  /* device int32 or NULL                                           */
 } ssn_codec_t;
 
 /*
@@ -130,8 +143,8 @@ ssn_status_t ssn_compress(const ssn_codec_t *codec, const void *X, int64_t ldx,
                           void *stream);
 
 /*
- * Receiver side of Eq. (ssn_compress) ("the receiver reconstructs with U_k^T", and adds back
- * the PE and T_fixed it also holds):  Xhat[t,:] = Z[t,:] U^T + E[ids[t],:] + P[pos(t),:].
+ * Receiver side of Eq. (ssn_compress) (Sec. 4.1: the receiving stage expands with U_k^T and
+ * adds back the PE and T_fixed it also holds):  Xhat[t,:] = Z[t,:] U^T + E[ids[t],:] + P[pos(t),:].
  * With codec->E == NULL and codec->P == NULL this is the plain expansion Z U^T, which is also
  * how a receiving stage expands an incoming coefficient gradient.
  * Arguments as for ssn_compress with Z the input and Xhat [n_tokens x d] the output.
@@ -142,7 +155,8 @@ ssn_status_t ssn_decompress(const ssn_codec_t *codec, const void *Z, int64_t ldz
                             void *stream);
 
 /*
- * Backward pass ("the backward pass uses the same compression"; chain rule (grad L) U_k):
+ * Backward pass (Sec. 4.1, after Eq. ssn_compress: the activation gradient crosses the boundary
+ * compressed the same way; chain rule (grad L) U_k):
  *   mode & SSN_GRAD_COEFF:  dZ   [n_tokens x k] = G U           -- what crosses the link
  *   mode & SSN_GRAD_FULL :  Gpar [n_tokens x d] = (G U) U^T     -- the projected gradient
  * The coordinates are kept in fp32 between the two products of the FULL form.  E and P of the
@@ -153,9 +167,9 @@ ssn_status_t ssn_grad_project(const ssn_codec_t *codec, const void *G, int64_t l
                               void *Gpar, int64_t ldgp, void *stream);
 
 /*
- * Original-SSN weight re-projection ("projecting it back into the subspace after every
- * optimizer step", Sec. 4.1; done outside the autograd graph, ablation Sec. "Reparameterized
- * SSN"), in place, for a batch of equally shaped weights:
+ * Original-SSN weight re-projection (Sec. 4.1: each constrained projection is put back into
+ * the subspace after every optimizer step, outside the autograd graph; ablation Sec.
+ * "Reparameterized SSN"), in place, for a batch of equally shaped weights:
  *   SSN_SIDE_RIGHT: W is [rows x cols] with cols == d, the layout of Eq. (residual_stream)
  *                   whose ROWS must lie in span(U):      W <- (W U) U^T
  *   SSN_SIDE_LEFT : W is [rows x cols] with rows == d (the transposed storage):
@@ -212,9 +226,10 @@ ssn_status_t ssn_reparam_project(const ssn_codec_t *codec, const void *H, int64_
                                  int64_t ldy, void *coords, int64_t ldc, void *stream);
 
 /*
- * Gradient of a reparameterized projection's factor (the chain rule quoted with Eq. reparam:
- * "the gradient for Z is (grad_W L) U_k"): with Y = (H Zw) U^T and dY = dL/dY,
+ * Gradient of a reparameterized projection's factor (the chain rule stated with Eq. reparam:
+ * the factor's gradient is the weight gradient times U_k): with Y = (H Zw) U^T and dY = dL/dY,
  *     dZw [m x k] = H^T (dY U)        (fp32 output, written, not accumulated)
+ * n_tokens == 0 writes zeros (an empty sum).
  *   workspace  device scratch of n * kpad * sizeof(element) bytes, kpad = k rounded up to 8,
  *              16-byte aligned: the coordinates dY U (in the storage dtype).
  * E and P of the codec are not used.
@@ -225,15 +240,17 @@ ssn_status_t ssn_reparam_grad_factor(const ssn_codec_t *codec, const void *H, in
                                      size_t workspace_bytes, void *stream);
 
 /*
- * Head-stage input of the reparameterized SSN (Sec. 4.1: the trainable embedding is factored as
- * T_S = Elow U_k^T "with every projection and the embedding parameterized through U_k"):
+ * Head-stage input of the reparameterized SSN (Sec. 4.1, after Eq. reparam: the trainable
+ * embedding is factored through U_k as well, T_S = Elow U_k^T):
  *     X0[t,:] = E[ids[t],:] + Elow[ids[t],:] U^T + P[pos(t),:]
  * i.e. ssn_decompress applied to the gathered rows of Elow [vocab x k]; compressing X0 gives
  * those rows back exactly.
  *   workspace  device scratch of n * kpad * sizeof(element) bytes, kpad = k rounded up to 8,
  *              16-byte aligned: the gathered coordinates.
- * ids, pos, seq_len, dev_status as for ssn_decompress; an id outside the table contributes
- * neither of its two rows.  Elow rows are used whether or not the codec has E.
+ * ids, pos, seq_len, dev_status as for ssn_decompress.  Each table is checked against its own
+ * row count: an id outside [0, vocab_low) contributes no Elow row, an id outside
+ * [0, codec->vocab) no E row, and either sets SSN_DEV_BAD_ID.  Elow rows are used whether or
+ * not the codec has E.
  */
 ssn_status_t ssn_head_embed(const ssn_codec_t *codec, const void *Elow, int64_t ldel,
                             int64_t vocab_low, const int32_t *ids, const int32_t *pos,
@@ -258,9 +275,9 @@ ssn_status_t ssn_head_embed(const ssn_codec_t *codec, const void *Elow, int64_t 
  *                         the rows and the `ids` argument is ignored.  A bf16 codec with
  *                         2 * kpad <= 128 (kpad = k rounded up to 8) runs on the tensor cores
  *                         with the fp32 coordinates split into a bf16 head and a bf16 remainder
- *                         (rank 2 * kpad against the basis repeated twice), so no precision of
- *                         the coordinates is dropped before the single rounding of X^; for that
- *                         the call needs a 256-byte aligned workspace of
+ *                         (rank 2 * kpad against the basis repeated twice), which keeps about 16
+ *                         of the 24 significand bits of a coordinate, far below the single
+ *                         bf16 rounding of X^; for that the call needs a 256-byte aligned workspace of
  *                         ssn_decompress_wire_workspace_bytes() bytes.  With a smaller (or
  *                         misaligned) workspace the general kernel runs; with_ids always needs
  *                         at least n_tokens * 4 bytes (rounded up to 256).
@@ -342,6 +359,40 @@ int32_t ssn_version(void);
  * its launch count.
  */
 int64_t ssn_launch_count(void);
+
+/*
+ * Diagnostic: which kernel the calling thread's most recent codec launch used, as
+ * family | (variant bits << 8); SSN_KERNEL_NONE before the first launch.  No counterpart in
+ * the paper; the tests use it to assert that a shape reaches the kernel it is meant to check.
+ */
+enum {
+  SSN_KERNEL_NONE = 0,
+  SSN_KERNEL_GENERIC = 1,          /* fp32 FMA kernels: any dtype, shape and alignment         */
+  SSN_KERNEL_MMA_SYNC = 2,         /* mma.sync, whole rows per warp                            */
+  SSN_KERNEL_MMA_SYNC_DSPLIT = 3,  /* mma.sync, few rows per SM: the warps of a CTA split d    */
+  SSN_KERNEL_EXPAND64 = 4,         /* mma.sync expansion, 64-column chunks                     */
+  SSN_KERNEL_UMMA_PROJECT = 5,     /* tcgen05 + TMA projection                                 */
+  SSN_KERNEL_UMMA_EXPAND = 6,      /* tcgen05 + TMA expansion                                  */
+  SSN_KERNEL_UMMA_ROUNDTRIP = 7,   /* tcgen05 + TMA project-then-expand                        */
+  SSN_KERNEL_UMMA_TOKENS = 8       /* tcgen05 + TMA contraction over tokens                    */
+};
+#define SSN_KVAR_E 1      /* the kernel reads E rows                                            */
+#define SSN_KVAR_P 2      /* the kernel reads P rows                                            */
+#define SSN_KVAR_WIDE 4   /* rank above 64 (two 64-coordinate groups / the wide row tiles)      */
+#define SSN_KVAR_ALT 8    /* MMA_SYNC: 32 rows per warp; EXPAND64: one P row per 16-sequence tile;
+                             UMMA_PROJECT: positional product shared per block; UMMA_EXPAND:
+                             tiles of 8 sequences x 16 positions; UMMA_ROUNDTRIP: LEFT          */
+#define SSN_KVAR_ROWSUMSQ 16 /* UMMA_EXPAND / EXPAND64 / GENERIC: the row statistic is produced  */
+int32_t ssn_last_kernel(void);
+
+/*
+ * Self-test of the bounded waits (no counterpart in the paper).  Launches one tiny kernel that
+ * waits, with the same helper every tensor-core kernel uses, on a barrier nobody arrives on,
+ * for at most max_polls polls (1 <= max_polls <= 1 << 20); the wait gives up, the kernel ORs
+ * SSN_DEV_TIMEOUT into *dev_status (device int32, required) and ends normally.  Nothing hangs
+ * and the context stays usable; the call exists so that this path can be exercised at all.
+ */
+ssn_status_t ssn_selftest_bounded_wait(int32_t max_polls, int32_t *dev_status, void *stream);
 
 #ifdef __cplusplus
 }

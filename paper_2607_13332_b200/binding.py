@@ -20,7 +20,11 @@ SSN_ERR_NULL, SSN_ERR_SHAPE, SSN_ERR_DTYPE, SSN_ERR_WORKSPACE, SSN_ERR_CUDA = 1,
 SSN_F32, SSN_BF16 = 0, 1
 SSN_SIDE_LEFT, SSN_SIDE_RIGHT = 0, 1
 SSN_GRAD_COEFF, SSN_GRAD_FULL = 1, 2
-SSN_DEV_BAD_ID, SSN_DEV_BAD_POS = 1, 2
+SSN_DEV_BAD_ID, SSN_DEV_BAD_POS, SSN_DEV_TIMEOUT = 1, 2, 4
+# ssn_last_kernel(): family | variant bits << 8
+(SSN_KERNEL_NONE, SSN_KERNEL_GENERIC, SSN_KERNEL_MMA_SYNC, SSN_KERNEL_MMA_SYNC_DSPLIT, SSN_KERNEL_EXPAND64,
+ SSN_KERNEL_UMMA_PROJECT, SSN_KERNEL_UMMA_EXPAND, SSN_KERNEL_UMMA_ROUNDTRIP, SSN_KERNEL_UMMA_TOKENS) = range(9)
+SSN_KVAR_E, SSN_KVAR_P, SSN_KVAR_WIDE, SSN_KVAR_ALT, SSN_KVAR_ROWSUMSQ = 1, 2, 4, 8, 16
 
 DTYPES = {"f32": SSN_F32, "bf16": SSN_BF16}
 SIDES = {"left": SSN_SIDE_LEFT, "right": SSN_SIDE_RIGHT}
@@ -41,6 +45,7 @@ class ssn_codec_t(ctypes.Structure):
         ("P", ctypes.c_void_p), ("ldp", ctypes.c_int64),
         ("EU", ctypes.c_void_p), ("ldeu", ctypes.c_int64),
         ("PU", ctypes.c_void_p), ("ldpu", ctypes.c_int64),
+        ("dev_status", ctypes.c_void_p),
     ]
 
 
@@ -91,6 +96,8 @@ _SIGNATURES = {
     "ssn_status_string": (ctypes.c_char_p, [_i32]),
     "ssn_version": (_i32, []),
     "ssn_launch_count": (_i64, []),
+    "ssn_last_kernel": (_i32, []),
+    "ssn_selftest_bounded_wait": (_i32, [_i32, _vp, _vp]),
 }
 for _name, (_res, _args) in _SIGNATURES.items():
     _fn = getattr(_lib, _name)
@@ -121,14 +128,26 @@ def ssn_launch_count() -> int:
     return int(_lib.ssn_launch_count())
 
 
+def ssn_last_kernel():
+    """(family, variant bits) of the calling thread's most recent codec launch."""
+    code = int(_lib.ssn_last_kernel())
+    return code & 0xFF, code >> 8
+
+
+def ssn_selftest_bounded_wait(max_polls: int, dev_status: int, stream: int = 0) -> None:
+    """One tiny kernel whose bounded wait runs out: ORs SSN_DEV_TIMEOUT into *dev_status."""
+    _check(_lib.ssn_selftest_bounded_wait(max_polls, dev_status or None, stream or None),
+           "ssn_selftest_bounded_wait")
+
+
 def make_codec(d: int, k: int, dtype: int, U: int, ldu: Optional[int] = None, E: int = 0,
                lde: Optional[int] = None, vocab: int = 0, P: int = 0,
-               ldp: Optional[int] = None, max_pos: int = 0) -> ssn_codec_t:
+               ldp: Optional[int] = None, max_pos: int = 0, dev_status: int = 0) -> ssn_codec_t:
     """Fill an ``ssn_codec_t`` from raw device addresses (0 = NULL = term absent)."""
     return ssn_codec_t(d=d, k=k, dtype=dtype, max_pos=max_pos, U=U or None,
                        ldu=k if ldu is None else ldu, E=E or None,
                        lde=d if lde is None else lde, vocab=vocab, P=P or None,
-                       ldp=d if ldp is None else ldp)
+                       ldp=d if ldp is None else ldp, dev_status=dev_status or None)
 
 
 def _check(status: int, where: str) -> None:

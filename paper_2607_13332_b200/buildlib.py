@@ -6,16 +6,17 @@ import glob
 import os
 import shutil
 import subprocess
+from concurrent.futures import ThreadPoolExecutor
 
 PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG_DIR)
 CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "libssn.so")
 
-NVCC_FLAGS = [
-    "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-    "-Xcompiler", "-fPIC", "-shared", "-cudart", "static",
-]
+COMPILE_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
+                 "-Xcompiler", "-fPIC"]
+LINK_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-shared", "-cudart", "static"]
+OBJ_DIR = os.path.join(PKG_DIR, "build")
 
 
 def _nvcc() -> str:
@@ -30,7 +31,7 @@ def sources():
 
 
 def _inputs():
-    return (sources() + glob.glob(os.path.join(CSRC, "*.cuh"))
+    return (sources() + glob.glob(os.path.join(CSRC, "*.cuh")) + glob.glob(os.path.join(CSRC, "*.h"))
             + glob.glob(os.path.join(ROOT, "include", "*.h")) + [os.path.abspath(__file__)])
 
 
@@ -41,19 +42,38 @@ def is_stale() -> bool:
     return any(os.path.getmtime(p) > built for p in _inputs())
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    """Compile csrc/*.cu into libssn.so next to this file; returns the library path."""
-    if not force and not is_stale():
-        return LIB_PATH
-    cmd = [_nvcc()] + NVCC_FLAGS + ["-I", os.path.join(ROOT, "include"), "-I", CSRC]
+def _compile_one(src: str, verbose: bool):
+    """One translation unit -> object file (skipped when the object is newer than every input)."""
+    obj = os.path.join(OBJ_DIR, os.path.basename(src)[:-3] + ".o")
+    headers = [p for p in _inputs() if not p.endswith(".cu")]
+    if os.path.exists(obj) and all(os.path.getmtime(p) <= os.path.getmtime(obj) for p in [src] + headers):
+        return obj, ""
+    cmd = [_nvcc()] + COMPILE_FLAGS + ["-I", os.path.join(ROOT, "include"), "-I", CSRC]
     if verbose:
         cmd += ["-Xptxas", "-v"]
-    tmp = LIB_PATH + ".tmp"
-    cmd += ["-o", tmp] + sources()
-    proc = subprocess.run(cmd, capture_output=True, text=True)
+    proc = subprocess.run(cmd + ["-c", src, "-o", obj], capture_output=True, text=True)
     if proc.returncode != 0:
-        raise RuntimeError("nvcc failed:\n" + proc.stdout + proc.stderr)
+        raise RuntimeError(f"nvcc failed on {src}:\n" + proc.stdout + proc.stderr)
+    return obj, proc.stderr
+
+
+def build(force: bool = False, verbose: bool = False) -> str:
+    """Compile csrc/*.cu (in parallel, one object per file) and link libssn.so next to this file;
+    returns the library path."""
+    if not force and not is_stale():
+        return LIB_PATH
+    os.makedirs(OBJ_DIR, exist_ok=True)
+    if force:
+        for old in glob.glob(os.path.join(OBJ_DIR, "*.o")):
+            os.remove(old)
+    with ThreadPoolExecutor(max_workers=min(8, os.cpu_count() or 1)) as pool:
+        results = list(pool.map(lambda src: _compile_one(src, verbose), sources()))
+    tmp = LIB_PATH + ".tmp"
+    proc = subprocess.run([_nvcc()] + LINK_FLAGS + ["-o", tmp] + [obj for obj, _ in results],
+                          capture_output=True, text=True)
+    if proc.returncode != 0:
+        raise RuntimeError("link failed:\n" + proc.stdout + proc.stderr)
     os.replace(tmp, LIB_PATH)
     if verbose:
-        print(proc.stderr)
+        print("".join(log for _, log in results))
     return LIB_PATH

@@ -32,8 +32,9 @@ constexpr int kStages = 3;
 constexpr int kZeroRowBytes = 65536;
 
 // A row of zeros that stands in for the E / P row of a token that has none (absent table,
-// index out of range, row past the end of the batch).  Never written.
-__device__ __align__(128) unsigned char g_zero_row[kZeroRowBytes];
+// index out of range, row past the end of the batch).  Never written.  One copy per translation
+// unit that gathers rows.
+static __device__ __align__(128) unsigned char g_zero_row[kZeroRowBytes];
 
 
 // ---- small PTX wrappers --------------------------------------------------------------------

@@ -4,6 +4,8 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
+#include <atomic>
+
 #include "ssn_common.cuh"
 
 namespace ssn {
@@ -56,7 +58,36 @@ cudaError_t launch_codec_umma_roundtrip_list(const MmaArgs &a, const __nv_bfloat
 // output is zeroed on the stream first when several CTAs share a row block.
 cudaError_t launch_codec_umma_tokens(const __nv_bfloat16 *H, int64_t ldh, const __nv_bfloat16 *C, int64_t ldc,
                                      float *out, int64_t ldout, int64_t n, int32_t m, int32_t k,
-                                     int sm_count, cudaStream_t stream);
+                                     int32_t *dev_status, int sm_count, cudaStream_t stream);
+
+// The self-test of the bounded waits (see ssn_selftest_bounded_wait).
+cudaError_t launch_bounded_wait_selftest(int max_polls, int32_t *dev_status, cudaStream_t stream);
+
+// Adds to the process-wide launch counter behind ssn_launch_count().
+void count_launches(int launches);
+
+// Records the kernel a launch used for ssn_last_kernel(): an SSN_KERNEL_* family and SSN_KVAR_* bits.
+void note_kernel(int family, int variant);
+
+// cudaFuncAttributeMaxDynamicSharedMemorySize belongs to the current device's context: it is set
+// once per device (`done` holds one bit per device ordinal) and always for ordinals past 63.
+template <typename Kernel>
+cudaError_t allow_dynamic_smem(Kernel kernel, int smem, std::atomic<uint64_t> &done) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  const uint64_t bit = dev >= 0 && dev < 64 ? 1ull << dev : 0ull;
+  if (bit != 0 && (done.load(std::memory_order_acquire) & bit)) return cudaSuccess;
+  e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  if (e == cudaSuccess && bit != 0) done.fetch_or(bit, std::memory_order_release);
+  return e;
+}
+
+// The tcgen05 kernels one by one; each returns cudaErrorNotSupported, with nothing launched, for
+// shapes and alignments that are not its own (the conditions are stated at the definitions).
+cudaError_t launch_codec_umma_project(const MmaArgs &a, bool shift, int sm_count, cudaStream_t stream);
+cudaError_t launch_codec_umma_expand(const MmaArgs &a, bool shift, int sm_count, cudaStream_t stream);
+cudaError_t launch_codec_umma_roundtrip(const MmaArgs &a, int sm_count, cudaStream_t stream);
 
 // mode: 1 = project, 2 = expand, 3 = project then expand (shift must be false).
 cudaError_t launch_codec_mma(const MmaArgs &a, bool shift, int mode, int sm_count,

@@ -53,11 +53,11 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
 }
-// Waits for the phase with the given parity; gives up (returns false) after kWaitSpins polls.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+// Waits for the phase with the given parity; gives up (returns false) after `limit` polls.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int limit = kWaitSpins) {
   int spins = 0;
   while (!mbar_try_wait(bar, parity))
-    if (++spins > kWaitSpins) return false;
+    if (++spins > limit) return false;
   return true;
 }
 // The same with cluster-scope acquire: the phase was completed by arrivals from the peer CTA

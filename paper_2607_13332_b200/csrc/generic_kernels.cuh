@@ -122,6 +122,7 @@ struct GatherArgs {
   const int32_t *ids;
   int64_t ld_table, ld_out, n, rows;
   int32_t k, kpad;
+  int32_t *dev_status;   // nullable: SSN_DEV_BAD_ID when an id is outside [0, rows)
 };
 
 template <typename T>
@@ -132,7 +133,9 @@ __global__ void gather_rows_kernel(const GatherArgs a) {
   const int j = (int)(i - t * a.kpad);
   const int64_t id = a.ids[t];
   T v = from_f32<T>(0.f);
-  if (j < a.k && id >= 0 && id < a.rows) v = static_cast<const T *>(a.table)[id * a.ld_table + j];
+  const bool in_table = id >= 0 && id < a.rows;
+  if (j < a.k && in_table) v = static_cast<const T *>(a.table)[id * a.ld_table + j];
+  if (!in_table && j == 0 && a.dev_status) atomicOr(a.dev_status, SSN_DEV_BAD_ID);
   static_cast<T *>(a.out)[t * a.ld_out + j] = v;
 }
 
@@ -145,7 +148,9 @@ __global__ void gather_rows_2d_kernel(const GatherArgs a) {
   if (t >= a.n) return;
   const int64_t id = a.ids[t];
   T v = from_f32<T>(0.f);
-  if (j < a.k && id >= 0 && id < a.rows) v = static_cast<const T *>(a.table)[id * a.ld_table + j];
+  const bool in_table = id >= 0 && id < a.rows;
+  if (j < a.k && in_table) v = static_cast<const T *>(a.table)[id * a.ld_table + j];
+  if (!in_table && j == 0 && a.dev_status) atomicOr(a.dev_status, SSN_DEV_BAD_ID);
   static_cast<T *>(a.out)[t * a.ld_out + j] = v;
 }
 

@@ -37,7 +37,7 @@ ssn_status_t make_shift(const ssn_codec_t *c, const int32_t *ids, const int32_t 
   s.vocab = c->vocab;
   s.max_pos = c->max_pos;
   s.seq_len = seq_len;
-  s.dev_status = dev_status;
+  s.dev_status = dev_status != nullptr ? dev_status : c->dev_status;
   if (c->E != nullptr) {
     if (ids == nullptr) return SSN_ERR_NULL;
     if (c->lde < c->d || c->vocab < 1) return SSN_ERR_SHAPE;
@@ -51,6 +51,7 @@ ssn_status_t make_shift(const ssn_codec_t *c, const int32_t *ids, const int32_t 
 }
 
 std::atomic<int64_t> g_launches{0};
+thread_local int32_t g_last_kernel = SSN_KERNEL_NONE;
 
 // Called after every group of `launches` kernel launches.
 ssn_status_t launch_status(int launches = 1) {
@@ -109,6 +110,9 @@ ssn_status_t launch_generic_token_kernel(const TokenArgs &a, int32_t dtype, cuda
     token_kernel<float><<<(unsigned)blocks, kGenericWarps * 32, smem, stream>>>(a);
   else
     token_kernel<__nv_bfloat16><<<(unsigned)blocks, kGenericWarps * 32, smem, stream>>>(a);
+  g_last_kernel = SSN_KERNEL_GENERIC |
+                  ((((a.sub_shift || a.add_shift) && a.shift.E ? SSN_KVAR_E : 0) |
+                    ((a.sub_shift || a.add_shift) && a.shift.P ? SSN_KVAR_P : 0)) << 8);
   return launch_status();
 }
 
@@ -155,6 +159,10 @@ ssn_status_t launch_token_kernel(const TokenArgs &a, int32_t dtype, cudaStream_t
 }
 
 }  // namespace
+
+void note_kernel(int family, int variant) { g_last_kernel = family | (variant << 8); }
+void count_launches(int launches) { g_launches.fetch_add(launches, std::memory_order_relaxed); }
+
 }  // namespace ssn
 
 namespace ssn {
@@ -174,6 +182,7 @@ ssn_status_t reproject_right_list(const ssn_codec_t *codec, void *const *W_ptrs,
       m.ldu = codec->ldu;
       m.d = codec->d;
       m.k = codec->k;
+      m.shift.dev_status = codec->dev_status;
       const __nv_bfloat16 *src[kMaxFusedMatrices];
       __nv_bfloat16 *dst[kMaxFusedMatrices];
       for (int32_t i = 0; i < take; ++i) src[i] = dst[i] = static_cast<__nv_bfloat16 *>(W_ptrs[done + i]);
@@ -199,6 +208,7 @@ ssn_status_t reproject_right_list(const ssn_codec_t *codec, void *const *W_ptrs,
         a.n = rows[b];
         a.d = codec->d;
         a.k = codec->k;
+        a.shift.dev_status = codec->dev_status;
         ssn_status_t st = launch_token_kernel(a, codec->dtype, s);
         if (st != SSN_OK) return st;
       }
@@ -224,6 +234,7 @@ bool try_reproject_left_fused(const ssn_codec_t *codec, void *const *W_ptrs, con
   m.ldu = codec->ldu;
   m.d = codec->d;
   m.k = codec->k;
+  m.shift.dev_status = codec->dev_status;
   const __nv_bfloat16 *src[kMaxFusedMatrices];
   __nv_bfloat16 *dst[kMaxFusedMatrices];
   for (int32_t i = 0; i < count; ++i) src[i] = dst[i] = static_cast<__nv_bfloat16 *>(W_ptrs[i]);
@@ -242,7 +253,7 @@ ssn_status_t reproject_left_general(const ssn_codec_t *codec, void *W, int64_t c
   if (workspace == nullptr || workspace_bytes < (size_t)codec->k * (size_t)cols * sizeof(float))
     return SSN_ERR_WORKSPACE;
   const int64_t col_blocks = (cols + kLeftCols - 1) / kLeftCols;
-  if (col_blocks > 0x7fffffffLL) return SSN_ERR_SHAPE;
+  if (col_blocks > 0x7fffffffLL || ((int64_t)codec->d + 31) / 32 > 65535) return SSN_ERR_SHAPE;
   LeftArgs a{};
   a.W = W;
   a.U = codec->U;
@@ -261,6 +272,7 @@ ssn_status_t reproject_left_general(const ssn_codec_t *codec, void *W, int64_t c
     left_reduce_kernel<__nv_bfloat16><<<g1, kLeftCols, 0, s>>>(a);
     left_expand_kernel<__nv_bfloat16><<<g2, kLeftCols, 0, s>>>(a);
   }
+  g_last_kernel = SSN_KERNEL_GENERIC;
   return launch_status(2);
 }
 
@@ -416,6 +428,7 @@ ssn_status_t ssn_grad_project(const ssn_codec_t *codec, const void *G, int64_t l
   a.n = n_tokens;
   a.d = codec->d;
   a.k = codec->k;
+  a.shift.dev_status = codec->dev_status;
   return launch_token_kernel(a, codec->dtype, static_cast<cudaStream_t>(stream));
 }
 
@@ -526,6 +539,7 @@ ssn_status_t ssn_grad_project_wire(const ssn_codec_t *codec, const void *G, int6
   a.n = n_tokens;
   a.d = codec->d;
   a.k = codec->k;
+  a.shift.dev_status = codec->dev_status;
   return launch_token_kernel(a, codec->dtype, static_cast<cudaStream_t>(stream));
 }
 
@@ -632,6 +646,7 @@ ssn_status_t ssn_reparam_project(const ssn_codec_t *codec, const void *H, int64_
     a.d1 = (int32_t)m;
     a.zout = static_cast<__nv_bfloat16 *>(coords);
     a.ldzout = ldc;
+    a.shift.dev_status = codec->dev_status;
     const __nv_bfloat16 *src = static_cast<const __nv_bfloat16 *>(H);
     __nv_bfloat16 *dst = static_cast<__nv_bfloat16 *>(Y);
     cudaError_t e = launch_codec_umma_roundtrip_list(a, &src, &dst, &n_tokens, &ldh, &ldy, 1, sms, s, false);
@@ -666,13 +681,19 @@ ssn_status_t ssn_reparam_grad_factor(const ssn_codec_t *codec, const void *H, in
                                      void *stream) {
   ssn_status_t st = check_codec(codec);
   if (st != SSN_OK) return st;
-  if (n_tokens < 1 || m < 1 || m > 0x7fffffffLL || ldh < m || lddy < codec->d || lddz < codec->k) return SSN_ERR_SHAPE;
-  if (H == nullptr || dY == nullptr || dZw == nullptr) return SSN_ERR_NULL;
+  if (n_tokens < 0 || m < 1 || m > 0x7fffffffLL || ldh < m || lddy < codec->d || lddz < codec->k) return SSN_ERR_SHAPE;
+  if (dZw == nullptr) return SSN_ERR_NULL;
+  if (n_tokens == 0) {   // an empty sum over the tokens
+    const cudaError_t e = cudaMemset2DAsync(dZw, (size_t)lddz * sizeof(float), 0, (size_t)codec->k * sizeof(float),
+                                            (size_t)m, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? SSN_OK : SSN_ERR_CUDA;
+  }
+  if (H == nullptr || dY == nullptr) return SSN_ERR_NULL;
   const int32_t kpad = (codec->k + 7) / 8 * 8;
   const size_t esz = codec->dtype == SSN_F32 ? sizeof(float) : sizeof(__nv_bfloat16);
   if (workspace == nullptr || workspace_bytes < (size_t)n_tokens * (size_t)kpad * esz) return SSN_ERR_WORKSPACE;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  TokenArgs p{};      // C = dY U: "the backward pass uses the same compression"
+  TokenArgs p{};      // C = dY U: the same projection as the backward pass of the boundary
   p.src = dY;
   p.lds = lddy;
   p.zout = workspace;
@@ -682,13 +703,14 @@ ssn_status_t ssn_reparam_grad_factor(const ssn_codec_t *codec, const void *H, in
   p.n = n_tokens;
   p.d = codec->d;
   p.k = codec->k;
+  p.shift.dev_status = codec->dev_status;
   st = launch_token_kernel(p, codec->dtype, s);
   if (st != SSN_OK) return st;
   const int sms = sm_count_of_current_device();
   if (codec->dtype == SSN_BF16 && sms > 0) {
     cudaError_t e = launch_codec_umma_tokens(static_cast<const __nv_bfloat16 *>(H), ldh,
                                              static_cast<const __nv_bfloat16 *>(workspace), kpad, dZw, lddz,
-                                             n_tokens, (int32_t)m, codec->k, sms, s);
+                                             n_tokens, (int32_t)m, codec->k, codec->dev_status, sms, s);
     if (e == cudaSuccess) {
       g_launches.fetch_add(1, std::memory_order_relaxed);
       return SSN_OK;
@@ -736,6 +758,7 @@ ssn_status_t ssn_head_embed(const ssn_codec_t *codec, const void *Elow, int64_t 
   g.rows = vocab_low;
   g.k = codec->k;
   g.kpad = kpad;
+  g.dev_status = dev_status != nullptr ? dev_status : codec->dev_status;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (kpad <= 256) {
     const int rows_per_block = 256 / (int)kpad;
@@ -825,5 +848,15 @@ const char *ssn_status_string(ssn_status_t status) {
 int32_t ssn_version(void) { return SSN_VERSION; }
 
 int64_t ssn_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+int32_t ssn_last_kernel(void) { return g_last_kernel; }
+
+ssn_status_t ssn_selftest_bounded_wait(int32_t max_polls, int32_t *dev_status, void *stream) {
+  if (dev_status == nullptr) return SSN_ERR_NULL;
+  if (max_polls < 1 || max_polls > (1 << 20)) return SSN_ERR_SHAPE;
+  const cudaError_t e = launch_bounded_wait_selftest(max_polls, dev_status, static_cast<cudaStream_t>(stream));
+  g_launches.fetch_add(1, std::memory_order_relaxed);
+  return e == cudaSuccess ? SSN_OK : SSN_ERR_CUDA;
+}
 
 }  // extern "C"

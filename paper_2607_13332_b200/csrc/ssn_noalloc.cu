@@ -5,6 +5,9 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
+#include <atomic>
+
+#include "codec_mma_launch.h"
 #include "generic_kernels.cuh"
 
 namespace ssn {
@@ -16,7 +19,7 @@ constexpr size_t kStaticScratchBytes = SSN_STATIC_SCRATCH_BYTES;
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
 
 constexpr int kMaxDevices = 64;
-float *g_scratch_ptr[kMaxDevices];   // device address of g_static_scratch, per device (0 = not set up)
+std::atomic<float *> g_scratch_ptr[kMaxDevices];   // device address of g_static_scratch, per device (0 = not set up)
 
 // The array's name is only a host-side handle; kernels need its device address, which the
 // runtime hands out per device (the device that is current when it is asked).
@@ -26,15 +29,17 @@ float *scratch_of_current_device() {
     cudaGetLastError();
     return nullptr;
   }
-  if (g_scratch_ptr[dev] == nullptr) {
+  float *known = g_scratch_ptr[dev].load(std::memory_order_acquire);
+  if (known == nullptr) {   // two threads may both ask; they get the same address
     void *p = nullptr;
     if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || p == nullptr) {
       cudaGetLastError();
       return nullptr;
     }
-    g_scratch_ptr[dev] = static_cast<float *>(p);
+    known = static_cast<float *>(p);
+    g_scratch_ptr[dev].store(known, std::memory_order_release);
   }
-  return g_scratch_ptr[dev];
+  return known;
 }
 
 }  // namespace
@@ -56,7 +61,8 @@ ssn_status_t ssn_weight_reproject_left_static(const ssn_codec_t *codec, void *W,
   // the fixed scratch must hold k x cols fp32 coordinates
   if ((size_t)codec->k * (size_t)cols > kStaticScratchBytes / sizeof(float)) return SSN_ERR_WORKSPACE;
   const int64_t col_blocks = (cols + kLeftCols - 1) / kLeftCols;
-  if (col_blocks > 0x7fffffffLL) return SSN_ERR_SHAPE;
+  // both kernels' grids must be launchable before the first one runs
+  if (col_blocks > 0x7fffffffLL || ((int64_t)codec->d + 31) / 32 > 65535) return SSN_ERR_SHAPE;
   float *scratch = scratch_of_current_device();
   if (scratch == nullptr) return SSN_ERR_CUDA;
 
@@ -79,6 +85,8 @@ ssn_status_t ssn_weight_reproject_left_static(const ssn_codec_t *codec, void *W,
     left_reduce_kernel<__nv_bfloat16><<<g1, kLeftCols, 0, s>>>(a);
     left_expand_kernel<__nv_bfloat16><<<g2, kLeftCols, 0, s>>>(a);
   }
+  count_launches(2);
+  note_kernel(SSN_KERNEL_GENERIC, 0);
   return cudaGetLastError() == cudaSuccess ? SSN_OK : SSN_ERR_CUDA;
 }
 

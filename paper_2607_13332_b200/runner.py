@@ -73,7 +73,7 @@ class Codec:
             E.data_ptr() if E is not None else 0, _ld(E) if E is not None else None,
             E.shape[0] if E is not None else 0,
             P.data_ptr() if P is not None else 0, _ld(P) if P is not None else None,
-            P.shape[0] if P is not None else 0)
+            P.shape[0] if P is not None else 0, dev_status=self.dev_status.data_ptr())
 
     def prepare_tables(self, embedding: bool = True, positions: bool = True) -> None:
         """Project the codec's constant tables once (EU = E U, PU = P U, fp32) and attach them,
@@ -101,10 +101,19 @@ class Codec:
         return torch.empty((rows, cols), dtype=_TORCH_DTYPE[self.dtype], device=self.U.device)
 
     def take_status(self) -> int:
-        """Read and clear the device status word (synchronises)."""
+        """Read and clear the device status word (synchronises): SSN_DEV_BAD_ID, SSN_DEV_BAD_POS
+        and SSN_DEV_TIMEOUT bits of every call made through this object since the last read."""
         v = int(self.dev_status.item())
         self.dev_status.zero_()
         return v
+
+    @staticmethod
+    def describe_status(status: int) -> str:
+        names = [name for bit, name in ((binding.SSN_DEV_BAD_ID, "token id outside the table"),
+                                        (binding.SSN_DEV_BAD_POS, "position outside the table"),
+                                        (binding.SSN_DEV_TIMEOUT, "a kernel's bounded wait ran out: output invalid"))
+                 if status & bit]
+        return "; ".join(names) if names else "ok"
 
     def compress(self, X: torch.Tensor, ids: Optional[torch.Tensor] = None, seq_len: int = 1,
                  pos: Optional[torch.Tensor] = None, out: Optional[torch.Tensor] = None) -> torch.Tensor:

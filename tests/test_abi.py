@@ -84,3 +84,41 @@ def test_binding_raises_with_a_message(libssn):
     with pytest.raises(libssn.SsnError) as err:
         libssn.ssn_compress(_codec(libssn), 0, 64, 0, 0, 4, 1, 0x2000, 8)
     assert err.value.status == libssn.SSN_ERR_NULL and "NULL" in str(err.value)
+
+
+def test_validation_from_two_threads_at_once(libssn):
+    """Host-side validation touches no shared state: two threads hammering it get the same codes."""
+    import threading
+
+    b = libssn
+    compress = b.raw("ssn_compress")
+    ok, bad = _codec(b), _codec(b, k=65)
+    results = [[], []]
+
+    def worker(slot):
+        for i in range(2000):
+            c = ok if (i + slot) % 2 == 0 else bad
+            results[slot].append(compress(ctypes.byref(c), 0x2000, 64, None, None, -1 if c is ok else 4, 1,
+                                          0x2000, 65, None, None))
+
+    threads = [threading.Thread(target=worker, args=(s,)) for s in (0, 1)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    for slot in (0, 1):
+        assert set(results[slot]) == {b.SSN_ERR_SHAPE} and len(results[slot]) == 2000
+
+
+def test_diagnostics_and_selftest_arguments(libssn):
+    b = libssn
+    fam, var = b.ssn_last_kernel()
+    assert 0 <= fam <= b.SSN_KERNEL_UMMA_TOKENS and var >= 0
+    selftest = b.raw("ssn_selftest_bounded_wait")
+    assert selftest(1000, None, None) == b.SSN_ERR_NULL
+    assert selftest(0, 0x1000, None) == b.SSN_ERR_SHAPE
+    assert selftest((1 << 20) + 1, 0x1000, None) == b.SSN_ERR_SHAPE
+    # the codec struct carries the optional status word as its last field
+    assert b.ssn_codec_t._fields_[-1][0] == "dev_status"
+    grad_factor = b.raw("ssn_reparam_grad_factor")
+    assert grad_factor(ctypes.byref(_codec(b)), None, 64, 64, None, 64, -1, 0x1000, 8, None, 0, None) == b.SSN_ERR_SHAPE

@@ -1,6 +1,9 @@
-"""GPU parity for the shapes that reach the tcgen05 kernels (large token counts, d a multiple of
-128, k <= 64 for the expansion kernels) and for the prepared tables EU = E U, PU = P U, each
-against the CPU oracle element by element."""
+"""GPU parity on batches of whole sequences at 512 to 8192 tokens, against the CPU oracle element
+by element.  At these sizes the projections (compress, grad-project) and the fused
+project-then-expand run on the tcgen05 kernels, while decompress takes the few-rows-per-SM
+mma.sync kernel; the tcgen05 expansion and the large-batch mma.sync kernels are covered, with an
+assertion of which kernel ran, in test_gpu_dispatch_coverage.py.  Also here: the prepared tables
+EU = E U, PU = P U, the re-projection lists, guard bands and odd leading dimensions."""
 
 import numpy as np
 import pytest
@@ -12,9 +15,7 @@ from tests.harness import Codec, assert_close, f64, guards_intact, host64, padde
 
 pytestmark = pytest.mark.gpu
 
-# batch, seq_len, d, k, vocab: batches of 8 whole sequences whose length is a multiple of 16
-# take the 8 x 16 tiles of the expansion kernel, the others its 128-token tiles or the
-# mma.sync kernel
+# batch, seq_len, d, k, vocab
 SHAPES = [
     (8, 128, 256, 40, 300),
     (32, 256, 1024, 40, 5000),
