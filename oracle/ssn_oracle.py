@@ -27,7 +27,9 @@ shapes; for the reparameterized forms (Eq. reparam): the materialised weight W_p
 membership of the subspace, loops, and the exact recovery of the factored embedding's coordinates
 by compress; for compress_sum: linearity against a loop-written R U and the exact recovery of
 summed coordinates; for the wire rows: IEEE-754 bit patterns typed by hand, the id word, the round trip
-within half an fp32 ulp.  No function here is left unpinned.
+within half an fp32 ulp; for decompress_rowsumsq: the hand-worked example's rows squared by hand,
+the closed form |Z|^2 + 2 <Z, s U> + |s|^2 for an orthonormal basis, loops, and the unit mean square
+of the row it normalises.  No function here is left unpinned.
 """
 
 from __future__ import annotations
@@ -93,6 +95,17 @@ def decompress(Z: np.ndarray, U: np.ndarray, E=None, ids=None, P=None, pos=None)
     U = np.asarray(U, dtype=np.float64)
     shift, status = shift_rows(Z.shape[0], U.shape[0], E, ids, P, pos)
     return Z @ U.T + shift, status
+
+
+def decompress_rowsumsq(Z: np.ndarray, U: np.ndarray, E=None, ids=None, P=None, pos=None):
+    """Receiver side fused with the row statistic of the receiving stage's first block: every
+    block of the paper's models opens with an RMSNorm (model table of the experimental setup),
+    whose only reduction is sum_i Xhat[t, i]^2 over the row that decompress has just produced
+    (Sec. 4.1 puts decompress first on the receiving stage).  Returns (Xhat [n, d], rowsumsq [n],
+    status); the squares are of the UNROUNDED reconstruction (the reading taken: the statistic is
+    formed before the single rounding of Xhat to its storage type)."""
+    Xhat, status = decompress(Z, U, E, ids, P, pos)
+    return Xhat, (Xhat * Xhat).sum(axis=1), status
 
 
 def grad_project_coeff(G: np.ndarray, U: np.ndarray) -> np.ndarray:

@@ -55,6 +55,38 @@ def test_hand_worked_grad_and_reproject():
     np.testing.assert_allclose(oracle.weight_reproject(R.T.copy(), U4, "left"), RP.T, atol=1e-15)
 
 
+def test_hand_worked_row_sum_of_squares():
+    # rows of XHAT4 squared by hand: 4+16+4+4, 2.25+1+2.25+0, 0+4+0+0
+    Xh, ss, status = oracle.decompress_rowsumsq(Z4, U4, E4, IDS4, P4, POS4)
+    assert status == 0
+    np.testing.assert_allclose(Xh, XHAT4, rtol=0, atol=1e-15)
+    np.testing.assert_allclose(ss, [28.0, 5.5, 4.0], rtol=0, atol=1e-14)
+
+
+def test_row_sum_of_squares_closed_form_loops_and_normalisation():
+    """For orthonormal U and shift s = E[id] + P[pos]:  |Z U^T + s|^2 = |Z|^2 + 2 <Z, s U> + |s|^2,
+    each term written with explicit loops; without a shift the statistic is |Z|^2 (isometry); and
+    dividing the row by sqrt(rowsumsq / d) leaves a unit mean square (what RMSNorm does with it)."""
+    rng = np.random.default_rng(12)
+    n, d, k, vocab, seq = 7, 12, 3, 5, 4
+    U = synth.subspace_basis(d, k, seed=12)
+    E, P = rng.standard_normal((vocab, d)), rng.standard_normal((seq, d))
+    Z = rng.standard_normal((n, k))
+    ids, pos = rng.integers(0, vocab, n), rng.integers(0, seq, n)
+    Xh, ss, _ = oracle.decompress_rowsumsq(Z, U, E, ids, P, pos)
+    for t in range(n):
+        shift = [E[ids[t]][i] + P[pos[t]][i] for i in range(d)]
+        zz = sum(Z[t][j] ** 2 for j in range(k))
+        cross = sum(Z[t][j] * sum(shift[i] * U[i][j] for i in range(d)) for j in range(k))
+        assert abs(ss[t] - (zz + 2 * cross + sum(v * v for v in shift))) < 1e-11
+        row = [sum(Z[t][j] * U[i][j] for j in range(k)) + shift[i] for i in range(d)]     # the definition, by loops
+        assert abs(ss[t] - sum(v * v for v in row)) < 1e-11
+        normed = Xh[t] / np.sqrt(ss[t] / d)
+        assert abs(float(np.mean(normed ** 2)) - 1.0) < 1e-12
+    _, ss0, _ = oracle.decompress_rowsumsq(Z, U)
+    np.testing.assert_allclose(ss0, [sum(Z[t][j] ** 2 for j in range(k)) for t in range(n)], rtol=1e-12)
+
+
 def test_positions_default_is_t_mod_seq_len():
     np.testing.assert_array_equal(oracle.token_positions(7, 3), [0, 1, 2, 0, 1, 2, 0])
     np.testing.assert_array_equal(oracle.token_positions(3, 2), POS4)
