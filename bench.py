@@ -38,14 +38,21 @@ METRIC = "ssn_codec_tokens_per_s"
 UNIT = "tokens/s"
 FALLBACK_HBM_GBS = 6650.0
 
-# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of ONE launch of each kernel on the
-# default workload, from the ncu captures summarised under profiles/; None where not captured.
-NCU_TRAFFIC_BYTES = {"compress": None, "decompress": 648.9e6, "grad_project": 540.2e6,
-                     "weight_reproject": 238.4e6}
-NCU_TRAFFIC_COMPRESS = {True: 550.5e6, False: 712.3e6}     # keyed by "prepared tables"
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "dram_traffic.json")
 
 
-REPROJECT_ROWS_COLS = ((4096, 4096), (14336, 4096))
+def recorded_traffic(config_name, default_size):
+    """DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) that an earlier ncu
+    capture of this same workload recorded, read from profiles/dram_traffic.json (written next to
+    the ncu summaries).  A recorded capture, not a measurement of this run; {} for any other
+    workload size."""
+    if not default_size:
+        return {}
+    try:
+        with open(TRAFFIC_FILE) as fh:
+            return json.load(fh).get(config_name, {})
+    except (OSError, ValueError):
+        return {}
 
 
 def parse_args():
@@ -54,14 +61,21 @@ def parse_args():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
-    ap.add_argument("--batch", type=int, default=None, help="sequences per microbatch (default 32)")
+    ap.add_argument("--config", choices=["stage8b", "mid"], default="stage8b",
+                    help="stage8b: the 8B-class stage boundary the metric is quoted on (d=4096, k=40, "
+                         "65536 tokens, Zipf ids); mid: d=2048, k=32, vocab 32000, 32768 tokens, uniform "
+                         "ids, re-projection of W [2048 x 8192] on the left")
+    ap.add_argument("--batch", type=int, default=None, help="sequences per microbatch (default: the config's)")
+    ap.add_argument("--sustain-seconds", type=float, default=2.0,
+                    help="length of the sustained run behind the clock_sensitivity object (0: skip it)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--tables", action="store_true",
                     help="the step's compress reads the prepared tables E U, P U instead of gathering "
                          "the E and P rows (the default step gathers; the table variant is always "
                          "timed beside it as compress_prepared_tables)")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
-    ap.add_argument("--sweep", choices=["compress", "reproject", "reparam", "wire", "dp"], default=None,
+    ap.add_argument("--sweep", choices=["compress", "reproject", "reparam", "wire", "dp", "small", "fusions"],
+                    default=None,
                     help="instead of the step: time the compress sweep (d, k, tokens) or the "
                          "re-projection sweep (k, weight shape, 32 layers); one JSON line per point")
     return ap.parse_args()
@@ -70,22 +84,35 @@ def parse_args():
 def workload(args):
     from paper_2607_13332_b200 import synth
 
-    wl = synth.STAGE_8B
+    wl = synth.WORKLOADS[args.config]
     if args.batch is not None:
         wl = wl.scaled(batch=args.batch)
     return wl
 
 
+def reproject_weights(wl):
+    """(side, [(rows, cols), ...]) of the step's weight re-projection: the 8B block's out-proj and
+    down-proj with the subspace on the columns, or the mid config's W [d x 8192] with it on the rows."""
+    if wl.name == "mid":
+        return "left", [(wl.d, 8192)]
+    return "right", [(4096, wl.d), (14336, wl.d)]
+
+
 def config_of(wl, world, tables=False):
+    side, shapes = reproject_weights(wl)
+    ids = f"Zipf({wl.zipf_s})" if wl.ids_law == "zipf" else "uniform"
+    title = "8B-class stage boundary" if wl.name == "stage8b" else f"{wl.name} codec"
     return {
         "compress_terms": "prepared tables EU=E.U, PU=P.U (fp32, made once before the timed region)"
                           if tables else "E and P rows gathered every step",
-        "workload": f"8B-class stage boundary: d={wl.d}, k={wl.k}, vocab={wl.vocab}, "
-                    f"{wl.batch}x{wl.seq_len}={wl.n_tokens} tokens, bf16, Zipf({wl.zipf_s}) ids; "
-                    "compress + decompress + grad-project + re-projection of one block's "
-                    "out-proj [4096x4096] and down-proj [14336x4096] per step",
+        "workload": f"{title}: d={wl.d}, k={wl.k}, vocab={wl.vocab}, "
+                    f"{wl.batch}x{wl.seq_len}={wl.n_tokens} tokens, bf16, {ids} ids; "
+                    "compress + decompress + grad-project + re-projection of "
+                    + " and ".join(f"[{r}x{c}]" for r, c in shapes) + f" ({side}) per step",
         "d": wl.d, "k": wl.k, "vocab": wl.vocab, "tokens_per_rank": wl.n_tokens,
-        "replicas": world, "l2": "inputs larger than L2 (X, G, E: 0.5-1 GB each)",
+        "replicas": world,
+        "l2": f"inputs larger than L2 (X, G: {wl.n_tokens * wl.d * 2 / 1e6:.0f} MB each, "
+              f"E: {wl.vocab * wl.d * 2 / 1e6:.0f} MB)",
     }
 
 
@@ -103,9 +130,9 @@ def algorithmic_bytes(wl, ids, step, tables=False):
         return n * d * b + shift + d * k * b + n * k * b
     if step == "grad_project":
         return n * d * b + d * k * b + n * k * b
-    if step == "weight_reproject":        # both weights of one block, read once and written once
-        rows = sum(r for r, _ in REPROJECT_ROWS_COLS)
-        return 2 * rows * d * b + 2 * d * k * b
+    if step == "weight_reproject":        # every weight read once and written once
+        _, shapes = reproject_weights(wl)
+        return 2 * sum(r * c for r, c in shapes) * b + 2 * d * k * b
     raise ValueError(step)
 
 
@@ -113,9 +140,11 @@ def algorithmic_bytes(wl, ids, step, tables=False):
 # CPU oracle leg (cpu_baseline of the GPU arm, and the whole of --impl reference)
 # ----------------------------------------------------------------------------------------------
 def oracle_tokens_per_s(wl, seconds, seed=0x5EED + 32):
-    """Times the oracle, as it stands, on a bounded sample of the step: `sample` tokens through
-    compress, decompress and grad-project plus the same fraction of the two weights' rows."""
-    from threadpoolctl import threadpool_info
+    """Times the oracle, as it stands, on a bounded SAMPLE of the step: `sample` tokens through
+    compress, decompress and grad-project plus the same fraction of the re-projected weights, on
+    all host threads numpy's BLAS uses and once more on one thread.  tokens/s of the full step is
+    extrapolated from the sample (every token, row and column is independent)."""
+    from threadpoolctl import threadpool_info, threadpool_limits
 
     from oracle import ssn_oracle as oracle
     from paper_2607_13332_b200 import synth
@@ -126,8 +155,10 @@ def oracle_tokens_per_s(wl, seconds, seed=0x5EED + 32):
     t = synth.codec_inputs(small, seed=seed)
     pos = oracle.token_positions(sample, wl.seq_len)
     P = synth.to_storage(synth.sinusoidal_positions(wl.seq_len, wl.d), wl.dtype)
-    w_rows = max(1, (4096 + 14336) * sample // wl.n_tokens)
-    W = synth.projection_weight(w_rows, wl.d, seed, wl.dtype)
+    side, shapes = reproject_weights(wl)
+    free_extent = sum(r if side == "right" else c for r, c in shapes)
+    w_extent = max(1, free_extent * sample // wl.n_tokens)
+    W = synth.projection_weight(w_extent, wl.d, seed, wl.dtype)     # [extent x d]; transposed for the left side
 
     f = lambda a: synth.to_f64(a, wl.dtype)
     U, E, Pf = f(t["U"]), f(t["E"]), f(P)      # the shared tables are set up once, untimed
@@ -136,22 +167,31 @@ def oracle_tokens_per_s(wl, seconds, seed=0x5EED + 32):
         Z, _ = oracle.compress(f(t["X"]), U, E, t["ids"], Pf, pos)
         oracle.decompress(Z, U, E, t["ids"], Pf, pos)
         oracle.grad_project_coeff(f(t["G"]), U)
-        oracle.weight_reproject(f(W), U, "right")
+        Wf = f(W)
+        oracle.weight_reproject(Wf if side == "right" else np.ascontiguousarray(Wf.T), U, side)
 
-    one_pass()
-    t0 = time.perf_counter()
-    one_pass()
-    per_pass = time.perf_counter() - t0
-    reps = max(1, int(seconds / max(per_pass, 1e-3)))
-    t0 = time.perf_counter()
-    for _ in range(reps):
+    def rate(budget):
         one_pass()
-    elapsed = time.perf_counter() - t0
+        t0 = time.perf_counter()
+        one_pass()
+        per_pass = time.perf_counter() - t0
+        reps = max(1, int(budget / max(per_pass, 1e-3)))
+        t0 = time.perf_counter()
+        for _ in range(reps):
+            one_pass()
+        elapsed = time.perf_counter() - t0
+        return sample * reps / elapsed, reps, elapsed
+
+    value, reps, elapsed = rate(seconds)
     cores = max([i.get("num_threads", 1) for i in threadpool_info()] or [1])
+    with threadpool_limits(limits=1):
+        value_1, _, _ = rate(max(1.0, seconds / 4))
     return {
-        "value": sample * reps / elapsed, "unit": UNIT, "cores": int(cores), "kind": "oracle",
-        "sample": f"{reps} passes over {sample} tokens (+{w_rows} weight rows) of the step, "
-                  f"numpy fp64, {elapsed:.1f} s",
+        "value": value, "unit": UNIT, "cores": int(cores), "kind": "oracle", "extrapolated": True,
+        "value_1_thread": value_1,
+        "sample": f"{reps} passes over a {sample}-token sample (+{w_extent} weight {'rows' if side == 'right' else 'columns'}) "
+                  f"of the step, numpy fp64, {elapsed:.1f} s; tokens/s of the full step extrapolated from "
+                  "the sample (tokens are independent)",
     }, elapsed / reps
 
 
@@ -261,6 +301,7 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
     wl = workload(args)
+    default_size = args.batch is None
     dt = wl.dtype
     t = synth.codec_inputs(wl, seed=0x5EED + 32 + 1000 * rank)
     codec = Codec(dt, to_device(t["U"], dt), to_device(t["E"], dt), to_device(t["P"], dt))
@@ -277,20 +318,21 @@ def run_ours(args):
     dZ = torch.empty_like(Z)
     Xh = torch.empty_like(X)
     Z_h, dZ_h = Z.cpu().pin_memory(), dZ.cpu().pin_memory()
+    side, shapes = reproject_weights(wl)
     weights = [to_device(synth.projection_weight(r, c, 0x5EED, dt, layer=i), dt)
-               for i, (r, c) in enumerate(synth.REPROJECT_SHAPES_8B.values())]
+               for i, (r, c) in enumerate(shapes)]
     del t["X"], t["G"], t["E"]
 
     stream = torch.cuda.current_stream()
-    kernel_events = []
 
-    def reproject():     # both projections of the block in one call (and one launch)
-        codec.weight_reproject_rows(weights)
+    def reproject():     # every weight of the step in one call (and one launch)
+        codec.weight_reproject_list(weights, side)
 
     calls = (("compress", lambda: compress_codec.compress(X, ids, seq_len=wl.seq_len, out=Z)),
              ("decompress", lambda: codec.decompress(Z, ids, seq_len=wl.seq_len, out=Xh)),
              ("grad_project", lambda: codec.grad_project(G, out=dZ)),
              ("weight_reproject", reproject))
+    kernel_events = []
 
     def step(record=False):
         for name, call in calls:
@@ -315,12 +357,20 @@ def run_ours(args):
         dist_util.barrier()
         torch.cuda.synchronize()
 
-    def timed(fn, steps, **kw):
+    def timed(fn, steps, per_step=None, **kw):
+        """Device time of `steps` calls of fn, max over ranks; per_step (a list) also receives one
+        event pair per call."""
         barrier()
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         a.record(stream)
         for _ in range(steps):
+            if per_step is not None:
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
             fn(**kw)
+            if per_step is not None:
+                e1.record(stream)
+                per_step.append((e0, e1))
         b.record(stream)
         barrier()
         return dist_util.max_over_ranks(a.elapsed_time(b), device="cuda")
@@ -332,11 +382,14 @@ def run_ours(args):
     t_begin = time.perf_counter()
     ms_total = timed(step, args.steps)
     launches = binding.ssn_launch_count() - launches0
-    # same loop once more with events around every call (events add small gaps, so this pass
-    # is not the one that gives `value`)
+    # the same loop with an event pair around every step (median / min), then around every call
+    # (events add small gaps, so neither pass is the one that gives `value`)
+    step_events = []
+    timed(step, args.steps, per_step=step_events)
+    step_ms = sorted(a.elapsed_time(b) for a, b in step_events)
     timed(step, args.steps, record=True)
-    kernel_ms = {name: float(np.mean([a.elapsed_time(b) for n_, a, b in kernel_events if n_ == name]))
-                 for name, _ in calls}
+    per_call = {name: sorted(a.elapsed_time(b) for n_, a, b in kernel_events if n_ == name) for name, _ in calls}
+    kernel_ms = {name: float(np.mean(v)) for name, v in per_call.items()}
     # the compress variant that is not in the step, timed alone the same way
     other = codec if tables else codec_t
     other_name = "compress_rows" if tables else "compress_prepared_tables"
@@ -345,8 +398,21 @@ def run_ours(args):
         e2e_step()
     ms_e2e = timed(e2e_step, args.steps)
     t_end = time.perf_counter()
-    # the clock record spans all three timed passes (device-resident, per-kernel, end to end)
+    # the clock record spans all the timed passes above (device-resident, per-step, per-kernel, end to end)
     clocks = sampler.stop(t_begin, t_end) if sampler else None
+
+    # host time of one enqueue (argument marshalling, tensor maps, launch): 1000 calls, no device wait
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for _ in range(250):
+        step()
+    host_us_per_call = (time.perf_counter() - t0) / 1000 * 1e6
+    torch.cuda.synchronize()
+
+    sensitivity = None
+    if rank == 0 and world == 1 and args.sustain_seconds > 0:
+        sensitivity = clock_sensitivity(args, wl, calls, kernel_ms, clocks, local, timed)
+
     status = codec.take_status()
     status |= codec_t.take_status()
     if status != 0:
@@ -356,18 +422,21 @@ def run_ours(args):
         ms_per_step = ms_total / args.steps
         value = world * n / (ms_per_step * 1e-3)
         peak, peak_kind = measured_hbm_peak()
+        traffic = recorded_traffic(wl.name, default_size)
         kernels = {}
         for name, ms in kernel_ms.items():
             algo_k = algorithmic_bytes(wl, t["ids"], name, tables)
             gbs = algo_k / (ms * 1e-3) / 1e9
-            kernels[name] = {"ms": ms, "algorithmic_bytes": algo_k, "achieved": gbs, "frac": gbs / peak,
-                             "traffic": NCU_TRAFFIC_COMPRESS[tables] if name == "compress"
-                             else NCU_TRAFFIC_BYTES.get(name)}
+            key = "compress_prepared_tables" if (name == "compress" and tables) else name
+            kernels[name] = {"ms": ms, "ms_median": float(np.median(per_call[name])), "ms_min": per_call[name][0],
+                             "algorithmic_bytes": algo_k, "achieved": gbs, "frac": gbs / peak,
+                             "frac_of_8TBps": gbs / 8000.0, "traffic": traffic.get(key)}
         algo_o = algorithmic_bytes(wl, t["ids"], "compress", not tables)
         kernels[other_name] = {"ms": other_ms, "algorithmic_bytes": algo_o,
                                "achieved": algo_o / (other_ms * 1e-3) / 1e9,
                                "frac": algo_o / (other_ms * 1e-3) / 1e9 / peak,
-                               "traffic": NCU_TRAFFIC_COMPRESS[not tables],
+                               "frac_of_8TBps": algo_o / (other_ms * 1e-3) / 1e9 / 8000.0,
+                               "traffic": traffic.get("compress" if tables else "compress_prepared_tables"),
                                "note": "not part of the step; back-to-back launches"}
         # the roofline object describes the call that takes the largest share of the step
         dominant = max(kernel_ms, key=kernel_ms.get)
@@ -376,24 +445,75 @@ def run_ours(args):
         d2h = Z_h.numel() * 2 + dZ_h.numel() * 2
         out = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": True,
+            "warmup": max(3, args.warmup), "ms_per_step": ms_per_step,
+            "ms_per_step_median": float(np.median(step_ms)), "ms_per_step_min": step_ms[0],
+            "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": config_of(wl, world, tables),
             "roofline": {"bound": "hbm", "kernel": "ssn_" + dominant, "achieved": achieved,
                          "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                         "frac_of_8TBps": achieved / 8000.0,
                          "peak_kind": peak_kind, "algorithmic_bytes": algo,
                          "kernel_ms": kernel_ms[dominant], "traffic": kernels[dominant]["traffic"],
+                         "traffic_source": "recorded ncu capture of this workload (profiles/dram_traffic.json)"
+                                           if kernels[dominant]["traffic"] else None,
                          "kernels": kernels},
             "e2e": {"value": world * n / (ms_e2e / args.steps * 1e-3), "unit": UNIT,
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
             "gpu_launches": int(launches),
+            "host_us_per_call": host_us_per_call,
             "clocks": clocks,
         }
+        if sensitivity is not None:
+            out["clock_sensitivity"] = sensitivity
         if world == 1 and not args.no_cpu_baseline:
             out["cpu_baseline"], _ = oracle_tokens_per_s(wl, args.cpu_seconds)
         print(json.dumps(out))
     if world > 1:
         dist.destroy_process_group()
+
+
+def clock_sensitivity(args, wl, calls, burst_ms, burst_clocks, gpu_index, timed):
+    """How the step and each call depend on the SM clock, with the clocks the box gives (none is
+    set here).  The timed region of the bench lasts milliseconds and sees the boost clock; a run of
+    `--sustain-seconds` of back-to-back steps, and then of each call alone, sees whatever clock the
+    power cap leaves.  For each: time, median SM MHz while it ran, and their product (thousands
+    of SM clocks per launch).  A call whose product stays put while its time grows is bound on the
+    SM side (issue, shared memory); one whose time stays put is bound by HBM."""
+    import torch
+
+    def sustained(fn, seconds, block=None):
+        fn()
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        fn()
+        torch.cuda.synchronize()
+        once = max(time.perf_counter() - t0, 1e-5)
+        block = block or max(10, int(seconds / 20 / once))
+        sampler = ClockSampler(gpu_index)
+        time.sleep(0.05)
+        t_begin = time.perf_counter()
+        blocks = [timed(fn, block) / block for _ in range(20)]
+        t_end = time.perf_counter()
+        clocks = sampler.stop(t_begin, t_end)
+        return {"ms_median": float(np.median(blocks)), "ms_min": float(min(blocks)), "launches_per_block": block,
+                "blocks": 20, "sm_mhz": clocks["sm_mhz"], "reasons": clocks["reasons"],
+                "seconds": round(t_end - t_begin, 2)}
+
+    def step():
+        for _, call in calls:
+            call()
+
+    out = {"burst_sm_mhz": burst_clocks["sm_mhz"] if burst_clocks else None,
+           "step": sustained(step, args.sustain_seconds), "kernels": {}}
+    for name, call in calls:
+        r = sustained(call, max(0.4, args.sustain_seconds / 4))
+        mhz, burst_mhz = r["sm_mhz"], (burst_clocks or {}).get("sm_mhz")
+        r["kclocks_sustained"] = r["ms_median"] * mhz if mhz else None
+        r["burst_ms"] = burst_ms[name]
+        r["kclocks_burst"] = burst_ms[name] * burst_mhz if burst_mhz else None
+        out["kernels"][name] = r
+    return out
 
 
 def run_sweep(args):
@@ -424,17 +544,21 @@ def run_sweep(args):
         return a.elapsed_time(b) * 1e3 / reps
 
     if args.sweep == "compress":
+        # every point's output is compared with the oracle on sampled tokens by
+        # tests/test_gpu_sweep_parity.py, which draws the same inputs from synth_device
+        from paper_2607_13332_b200 import synth_device
         for d in (1024, 2048, 4096, 8192):
-            E = (torch.randn((vocab, d), device="cuda", generator=gen) * 0.02).bfloat16()
-            P = to_device(synth.to_storage(synth.sinusoidal_positions(seq, d), dt), dt)
+            gen = synth_device.generator(d)
+            E = synth_device.embedding_table(vocab, d, gen)
+            P = synth_device.positions_table(seq, d)
             for k in (8, 32, 64, 128):
-                U = to_device(synth.to_storage(synth.subspace_basis(d, k, 1), dt), dt)
+                U = synth_device.basis(d, k, 1)
                 codec, codec_t = Codec(dt, U, E, P), Codec(dt, U, E, P)
                 codec_t.prepare_tables()
                 for n in (4096, 65536, 524288):
-                    ids_np = np.random.default_rng(n + d + k).integers(0, vocab, n).astype(np.int32)
+                    ids_np = synth_device.uniform_ids(n, vocab, n + d + k)
                     ids = torch.from_numpy(ids_np).cuda()
-                    X = torch.randn((n, d), device="cuda", generator=gen).bfloat16()
+                    X = synth_device.activations(n, d, gen)
                     Z = torch.empty((n, k), dtype=torch.bfloat16, device="cuda")
                     uniq = int(np.unique(ids_np).size)
                     reps = 20 if n <= 65536 else 5
@@ -445,11 +569,84 @@ def run_sweep(args):
                         us = timed_us(lambda: c.compress(X, ids, seq_len=seq, out=Z), reps)
                         out[name] = {"us": round(us, 1), "GBps": round(algo / us / 1e3, 0),
                                      "frac_of_measured": round(algo / us / 1e3 / peak, 3)}
-                    status = codec.take_status() | codec_t.take_status()
-                    out["status"] = status
+                    out["status"] = Codec.describe_status(codec.take_status() | codec_t.take_status())
                     print(json.dumps(out), flush=True)
                     del X, Z, ids
             del E, P
+    elif args.sweep == "small":
+        # the call sizes of the paper's per-stage timing table (1 to 3 coalesced sequences of 4096
+        # tokens per call) at the 8B-class boundary; several input sets are rotated so that L2 does
+        # not hold a call's input from the call before; host_us is the enqueue cost of one call
+        from paper_2607_13332_b200 import synth_device
+        d, k = 4096, 40
+        gen = synth_device.generator(1)
+        E = synth_device.embedding_table(vocab, d, gen)
+        P = synth_device.positions_table(seq, d)
+        U = synth_device.basis(d, k, 1)
+        codec, codec_t = Codec(dt, U, E, P), Codec(dt, U, E, P)
+        codec_t.prepare_tables()
+        for n in (4096, 8192, 12288, 16384):
+            ids_np = synth.zipf_ids(n, vocab, 1.1, seed=n)
+            ids = torch.from_numpy(ids_np).cuda()
+            uniq = int(np.unique(ids_np).size)
+            nset = max(2, (512 << 20) // (n * d * 2))
+            Xs = [synth_device.activations(n, d, gen) for _ in range(nset)]
+            Zs = [synth_device.activations(n, k, gen) for _ in range(nset)]
+            Xh = torch.empty((n, d), dtype=torch.bfloat16, device="cuda")
+            Zo = torch.empty((n, k), dtype=torch.bfloat16, device="cuda")
+            turn = [0]
+
+            def nxt(sets):
+                turn[0] += 1
+                return sets[turn[0] % nset]
+
+            rows_bytes = n * d * 2 + uniq * d * 2 + min(seq, n) * d * 2 + d * k * 2 + n * k * 2
+            for name, fn, algo in (
+                    ("compress (rows)", lambda: codec.compress(nxt(Xs), ids, seq_len=seq, out=Zo), rows_bytes),
+                    ("compress (prepared tables)", lambda: codec_t.compress(nxt(Xs), ids, seq_len=seq, out=Zo),
+                     n * d * 2 + n * 4 + (uniq + min(seq, n)) * k * 4 + d * k * 2 + n * k * 2),
+                    ("grad_project", lambda: codec.grad_project(nxt(Xs), out=Zo), n * d * 2 + d * k * 2 + n * k * 2),
+                    ("decompress", lambda: codec.decompress(nxt(Zs), ids, seq_len=seq, out=Xh), rows_bytes)):
+                us = timed_us(fn, 40)
+                fam, var = binding.ssn_last_kernel()
+                t0 = time.perf_counter()
+                for _ in range(200):
+                    fn()
+                host_us = (time.perf_counter() - t0) / 200 * 1e6
+                torch.cuda.synchronize()
+                print(json.dumps({"sweep": "small", "op": name, "tokens": n, "d": d, "k": k, "us": round(us, 1),
+                                  "host_us": round(host_us, 1), "GBps": round(algo / us / 1e3, 0),
+                                  "frac_of_measured": round(algo / us / 1e3 / peak, 3),
+                                  "kernel_family": fam, "kernel_variant": var}), flush=True)
+            del Xs, Zs, Xh
+    elif args.sweep == "fusions":
+        # decompress with the RMSNorm row statistic of the receiving block, against decompress
+        # followed by a separate reduction over the rows it wrote (a library reduction stands in for
+        # the norm's first pass)
+        from paper_2607_13332_b200 import synth_device
+        d, k, n = 4096, 40, 65536
+        gen = synth_device.generator(2)
+        E = synth_device.embedding_table(vocab, d, gen)
+        P = synth_device.positions_table(seq, d)
+        codec = Codec(dt, synth_device.basis(d, k, 1), E, P)
+        ids_np = synth.token_ids(synth.STAGE_8B, 3)
+        ids = torch.from_numpy(ids_np).cuda()
+        uniq = int(np.unique(ids_np).size)
+        Z = synth_device.activations(n, k, gen)
+        Xh = torch.empty((n, d), dtype=torch.bfloat16, device="cuda")
+        ss = torch.empty(n, dtype=torch.float32, device="cuda")
+        algo = n * k * 2 + n * 4 + uniq * d * 2 + seq * d * 2 + d * k * 2 + n * d * 2
+        for name, fn, extra in (
+                ("decompress", lambda: codec.decompress(Z, ids, seq_len=seq, out=Xh), 0),
+                ("decompress_rowsumsq (fused)",
+                 lambda: codec.decompress_rowsumsq(Z, ids, seq_len=seq, out=Xh, rowsumsq=ss), n * 4),
+                ("decompress, then a separate sum of squares over Xhat",
+                 lambda: (codec.decompress(Z, ids, seq_len=seq, out=Xh), torch.linalg.vector_norm(Xh, dim=1, dtype=torch.float32, out=ss)),
+                 n * 4)):
+            us = timed_us(fn, 10)
+            print(json.dumps({"sweep": "fusions", "op": name, "tokens": n, "d": d, "k": k, "us": round(us, 1),
+                              "GBps": round((algo + extra) / us / 1e3, 0),
+                              "frac_of_measured": round((algo + extra) / us / 1e3 / peak, 3)}), flush=True)
     elif args.sweep == "reparam":
         # reparameterized SSN (Eq. reparam): Y = (H Zw) U^T for the block's two output projections,
         # and the head-stage input with the factored embedding, at the benchmark's token count

@@ -155,6 +155,28 @@ ssn_status_t ssn_decompress(const ssn_codec_t *codec, const void *Z, int64_t ldz
                             void *stream);
 
 /*
+ * ssn_decompress fused with the row statistic of the receiving stage's first block.  Sec. 4.1
+ * makes decompress the first operation of a receiving stage, and every block of the paper's
+ * models opens with an RMSNorm (model table of the experimental setup), whose only reduction
+ * over the row is
+ *     rowsumsq[t] = sum_i Xhat[t,i]^2
+ * so producing it here leaves the norm a pure scale of Xhat (no second pass over the row).
+ *   rowsumsq  device fp32 [n_tokens], written (the call zeroes it on the stream first).  The
+ *             squares are of the fp32 values BEFORE Xhat is rounded to the storage type; for
+ *             bf16 storage they differ from the squares of the stored row by ~2^-9 / sqrt(d)
+ *             relative.  Partial sums of a row are combined with atomic adds, so the last
+ *             bits may differ from run to run.
+ * Everything else as for ssn_decompress.  Performance note: the tensor-core expansion kernel
+ * produces the statistic for bf16 codecs with d a multiple of 128, k <= 128, at least 512
+ * tokens and, when the codec has P, implicit positions over groups of 8 whole sequences whose
+ * length is a multiple of 16; other calls run the general kernel.
+ */
+ssn_status_t ssn_decompress_rowsumsq(const ssn_codec_t *codec, const void *Z, int64_t ldz,
+                                     const int32_t *ids, const int32_t *pos, int64_t n_tokens,
+                                     int32_t seq_len, void *Xhat, int64_t ldx, float *rowsumsq,
+                                     int32_t *dev_status, void *stream);
+
+/*
  * Backward pass (Sec. 4.1, after Eq. ssn_compress: the activation gradient crosses the boundary
  * compressed the same way; chain rule (grad L) U_k):
  *   mode & SSN_GRAD_COEFF:  dZ   [n_tokens x k] = G U           -- what crosses the link

@@ -66,6 +66,7 @@ _codec_p = ctypes.POINTER(ssn_codec_t)
 _SIGNATURES = {
     "ssn_compress": (_i32, [_codec_p, _vp, _i64, _vp, _vp, _i64, _i32, _vp, _i64, _vp, _vp]),
     "ssn_decompress": (_i32, [_codec_p, _vp, _i64, _vp, _vp, _i64, _i32, _vp, _i64, _vp, _vp]),
+    "ssn_decompress_rowsumsq": (_i32, [_codec_p, _vp, _i64, _vp, _vp, _i64, _i32, _vp, _i64, _vp, _vp, _vp]),
     "ssn_grad_project": (_i32, [_codec_p, _vp, _i64, _i64, _i32, _vp, _i64, _vp, _i64, _vp]),
     "ssn_weight_reproject_workspace_bytes": (_sz, [_codec_p, _i64, _i64, _i32, _i32]),
     "ssn_weight_reproject": (_i32, [_codec_p, ctypes.POINTER(_vp), _i32, _i64, _i64, _i64, _i32,
@@ -167,6 +168,15 @@ def ssn_decompress(codec: ssn_codec_t, Z: int, ldz: int, ids: int, pos: int, n_t
     _check(_lib.ssn_decompress(ctypes.byref(codec), Z or None, ldz, ids or None, pos or None,
                                n_tokens, seq_len, Xhat or None, ldx, dev_status or None,
                                stream or None), "ssn_decompress")
+
+
+def ssn_decompress_rowsumsq(codec: ssn_codec_t, Z: int, ldz: int, ids: int, pos: int, n_tokens: int,
+                            seq_len: int, Xhat: int, ldx: int, rowsumsq: int, dev_status: int = 0,
+                            stream: int = 0) -> None:
+    """ssn_decompress that also writes rowsumsq[t] = sum_i Xhat[t,i]^2 (fp32, before rounding)."""
+    _check(_lib.ssn_decompress_rowsumsq(ctypes.byref(codec), Z or None, ldz, ids or None, pos or None,
+                                        n_tokens, seq_len, Xhat or None, ldx, rowsumsq or None,
+                                        dev_status or None, stream or None), "ssn_decompress_rowsumsq")
 
 
 def ssn_grad_project(codec: ssn_codec_t, G: int, ldg: int, n_tokens: int, mode: int, dZ: int = 0,

@@ -155,6 +155,9 @@ cudaError_t launch_codec_mma(const MmaArgs &a, bool shift, int mode, int sm_coun
   }
   // wire rows and a second addend: only the tcgen05 projection takes them
   if (a.zout32 != nullptr || a.src2 != nullptr) return cudaErrorNotSupported;
+  // the row statistic: only the tcgen05 expansion produces it, at any token count it takes
+  if (a.rowsumsq != nullptr)
+    return mode == kModeExpand ? launch_codec_umma_expand(a, shift, sm_count, stream) : cudaErrorNotSupported;
   if (mode == (kModeProject | kModeExpand) && !shift) {
     cudaError_t e = launch_codec_umma_roundtrip(a, sm_count, stream);
     if (e != cudaErrorNotSupported) return e;
@@ -162,6 +165,14 @@ cudaError_t launch_codec_mma(const MmaArgs &a, bool shift, int mode, int sm_coun
   const int nt = (a.k + 7) / 8;
   // With few tokens per warp a second 16-row tile would be computed for nothing.
   const bool small = a.n <= (int64_t)sm_count * kMmaWarps * 16;
+  // The tcgen05 expansion deals (tile, chunk) units to the SMs, so it fills the machine from 512
+  // tokens on; measured against the few-rows kernel it wins wherever the output is 8 MB or more,
+  // the model is wide or the rank needs the wide mma.sync tiles (16384 tokens, d = 4096: 48 us
+  // against 127 us), and loses a few microseconds of set-up on the smallest outputs.
+  if (small && mode == kModeExpand && (a.n * a.d >= (1 << 22) || a.d >= 2048 || nt > 8)) {
+    cudaError_t e = launch_codec_umma_expand(a, shift, sm_count, stream);
+    if (e != cudaErrorNotSupported) return e;
+  }
   if (small && nt <= 8) {
     // few rows per SM: the warps of a CTA share a row tile and split d
     return a.n > (int64_t)sm_count * 16 ? launch_dsplit<2>(a, shift, mode, nt, sm_count, stream)

@@ -34,6 +34,9 @@ struct MmaArgs {
   float *zout32;
   int64_t ldzout32;
   const int32_t *wire_ids;
+  // expansion with the row statistic: rowsumsq[t] += sum of squares of the fp32 output row t
+  // (zeroed by the caller); only the tcgen05 expansion takes it
+  float *rowsumsq;
   ShiftTables shift;
 };
 

@@ -347,10 +347,15 @@ codec_umma_expand_kernel(const MmaArgs a, const ExpandGeometry geo, const __grid
       const int s1 = geo.grid_mode ? c1 : c1 + quarter * 32;
       const int s2 = geo.grid_mode ? c2 + quarter * (32 / kGridPos) : 0;
       const bool rows_live = geo.grid_mode || (int64_t)s1 < a.n;
+      // this thread's token (row quarter * 32 + lane of the tile), for the row statistic
+      const int trow = quarter * 32 + lane;
+      const int64_t tok = geo.grid_mode ? (int64_t)(c2 + trow / kGridPos) * geo.seq_len + c1 + trow % kGridPos
+                                        : (int64_t)c1 + trow;
       int q0, q1;
       chunk_range(tile, q0, q1);
       for (int q = q0; q < q1; ++q, ++ccount) {
         if ((int)(ccount & 1) != group) continue;
+        float ss = 0.f;   // sum of squares of this row's 128 columns of the chunk, before rounding
         const int db = group;
         if (!dead && !mbar_wait(d_full_bar(db), (uint32_t)((ccount >> 1) & 1))) timed_out();
         asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
@@ -401,6 +406,8 @@ codec_umma_expand_kernel(const MmaArgs a, const ExpandGeometry geo, const __grid
                 f[2 * i + 1] += __uint_as_float(e[c][i] & 0xFFFF0000u);
               }
             }
+#pragma unroll
+            for (int i = 0; i < 8; ++i) ss = fmaf(f[i], f[i], ss);
             const uint32_t o0 = pack_bf16(f[0], f[1]), o1 = pack_bf16(f[2], f[3]);
             const uint32_t o2 = pack_bf16(f[4], f[5]), o3 = pack_bf16(f[6], f[7]);
             asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};\n" ::"r"(addr), "r"(o0), "r"(o1), "r"(o2), "r"(o3)
@@ -427,6 +434,7 @@ codec_umma_expand_kernel(const MmaArgs a, const ExpandGeometry geo, const __grid
           }
           held = g == kChunkCols / 64 - 1 ? -1 : eslot;
         }
+        if (a.rowsumsq != nullptr && tok < a.n) atomicAdd(a.rowsumsq + tok, ss);
       }
     }
     if (HAS_E && lane == 0) {

@@ -25,6 +25,7 @@ struct TokenArgs {
   // coordinates leave (zout, when projecting) or arrive (zin, when expanding) as fp32 words,
   // leading dimension in words; with wire_ids word k of an outgoing row is the token id
   int32_t wire, wire_ids;
+  float *rowsumsq;    // [n] sum of squares of the fp32 output row (before rounding), or nullptr
   int32_t sub_shift;  // phase 1 subtracts E[ids]+P[pos]   (Eq. ssn_compress)
   int32_t add_shift;  // phase 2 adds E[ids]+P[pos] back   (receiver side)
   ShiftTables shift;
@@ -102,6 +103,7 @@ token_kernel(const TokenArgs a) {
     const T *Ux = a.U2 != nullptr ? static_cast<const T *>(a.U2) : U;
     const int64_t ldux = a.U2 != nullptr ? a.ldu2 : a.ldu;
     const int dx = a.U2 != nullptr ? a.d2 : a.d;
+    float ss = 0.f;
     for (int i = lane; i < dx; i += 32) {
       const T *urow = Ux + (int64_t)i * ldux;
       float acc = 0.f;
@@ -110,7 +112,13 @@ token_kernel(const TokenArgs a) {
         if (erow) acc += to_f32(erow[i]);
         if (prow) acc += to_f32(prow[i]);
       }
+      ss = fmaf(acc, acc, ss);
       out[i] = from_f32<T>(acc);
+    }
+    if (a.rowsumsq != nullptr) {
+#pragma unroll
+      for (int off = 16; off > 0; off >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, off);
+      if (lane == 0) a.rowsumsq[t] = ss;
     }
   }
 }

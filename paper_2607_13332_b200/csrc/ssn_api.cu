@@ -112,7 +112,8 @@ ssn_status_t launch_generic_token_kernel(const TokenArgs &a, int32_t dtype, cuda
     token_kernel<__nv_bfloat16><<<(unsigned)blocks, kGenericWarps * 32, smem, stream>>>(a);
   g_last_kernel = SSN_KERNEL_GENERIC |
                   ((((a.sub_shift || a.add_shift) && a.shift.E ? SSN_KVAR_E : 0) |
-                    ((a.sub_shift || a.add_shift) && a.shift.P ? SSN_KVAR_P : 0)) << 8);
+                    ((a.sub_shift || a.add_shift) && a.shift.P ? SSN_KVAR_P : 0) |
+                    (a.rowsumsq != nullptr ? SSN_KVAR_ROWSUMSQ : 0)) << 8);
   return launch_status();
 }
 
@@ -120,7 +121,9 @@ ssn_status_t launch_token_kernel(const TokenArgs &a, int32_t dtype, cudaStream_t
   if (a.n == 0) return SSN_OK;
   // wire rows: the tensor-core path takes the projection only (and falls back when it refuses)
   const bool wire_ok = !(a.wire || a.src2) || (a.src != nullptr && a.dst == nullptr);
-  if (wire_ok && mma_eligible(a, dtype)) {
+  // the row statistic: only the plain expansion (no wire rows) on the tensor cores
+  const bool stat_ok = a.rowsumsq == nullptr || (a.src == nullptr && a.dst != nullptr && !a.wire);
+  if (wire_ok && stat_ok && mma_eligible(a, dtype)) {
     const int sms = sm_count_of_current_device();
     if (sms > 0) {
       MmaArgs m{};
@@ -137,6 +140,7 @@ ssn_status_t launch_token_kernel(const TokenArgs &a, int32_t dtype, cudaStream_t
       m.U = static_cast<const __nv_bfloat16 *>(a.U);
       m.src2 = static_cast<const __nv_bfloat16 *>(a.src2);
       m.lds2 = a.lds2;
+      m.rowsumsq = a.rowsumsq;
       m.lds = a.lds;
       m.ldzin = a.ldzin;
       m.ldzout = a.ldzout;
@@ -149,7 +153,7 @@ ssn_status_t launch_token_kernel(const TokenArgs &a, int32_t dtype, cudaStream_t
       const bool shift = (a.sub_shift || a.add_shift) && (a.shift.E || a.shift.P);
       const int mode = (a.src ? 1 : 0) | (a.dst ? 2 : 0);
       cudaError_t e = launch_codec_mma(m, shift, mode, sms, stream);
-      if (!((a.wire || a.src2) && e == cudaErrorNotSupported)) {
+      if (!((a.wire || a.src2 || a.rowsumsq) && e == cudaErrorNotSupported)) {
         g_launches.fetch_add(1, std::memory_order_relaxed);
         return e == cudaSuccess ? SSN_OK : SSN_ERR_CUDA;
       }
@@ -397,6 +401,38 @@ ssn_status_t ssn_decompress(const ssn_codec_t *codec, const void *Z, int64_t ldz
   a.k = codec->k;
   a.add_shift = 1;
   return launch_token_kernel(a, codec->dtype, static_cast<cudaStream_t>(stream));
+}
+
+ssn_status_t ssn_decompress_rowsumsq(const ssn_codec_t *codec, const void *Z, int64_t ldz,
+                                     const int32_t *ids, const int32_t *pos, int64_t n_tokens,
+                                     int32_t seq_len, void *Xhat, int64_t ldx, float *rowsumsq,
+                                     int32_t *dev_status, void *stream) {
+  ssn_status_t st = check_codec(codec);
+  if (st != SSN_OK) return st;
+  if (n_tokens < 0 || ldx < codec->d || ldz < codec->k) return SSN_ERR_SHAPE;
+  if (n_tokens == 0) return SSN_OK;
+  if (Xhat == nullptr || Z == nullptr || rowsumsq == nullptr) return SSN_ERR_NULL;
+  TokenArgs a{};
+  st = make_shift(codec, ids, pos, seq_len, dev_status, &a.shift);
+  if (st != SSN_OK) return st;
+  a.zin = Z;
+  a.ldzin = ldz;
+  a.dst = Xhat;
+  a.lddst = ldx;
+  a.U = codec->U;
+  a.ldu = codec->ldu;
+  a.n = n_tokens;
+  a.d = codec->d;
+  a.k = codec->k;
+  a.add_shift = 1;
+  a.rowsumsq = rowsumsq;
+  // the tensor-core kernel adds per-chunk partial sums atomically: start from zero
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (cudaMemsetAsync(rowsumsq, 0, (size_t)n_tokens * sizeof(float), s) != cudaSuccess) {
+    cudaGetLastError();
+    return SSN_ERR_CUDA;
+  }
+  return launch_token_kernel(a, codec->dtype, s);
 }
 
 ssn_status_t ssn_grad_project(const ssn_codec_t *codec, const void *G, int64_t ldg,

@@ -133,6 +133,18 @@ class Codec:
                                _ld(Xh), self.dev_status.data_ptr(), _stream())
         return Xh
 
+    def decompress_rowsumsq(self, Z: torch.Tensor, ids: Optional[torch.Tensor] = None, seq_len: int = 1,
+                            pos: Optional[torch.Tensor] = None, out: Optional[torch.Tensor] = None,
+                            rowsumsq: Optional[torch.Tensor] = None):
+        """decompress plus the RMSNorm statistic of the rows it writes: (Xhat, sum_i Xhat[t,i]^2)."""
+        n = Z.shape[0]
+        Xh = out if out is not None else self._empty(n, self.d)
+        ss = rowsumsq if rowsumsq is not None else torch.empty(n, dtype=torch.float32, device=self.U.device)
+        binding.ssn_decompress_rowsumsq(self.c, Z.data_ptr(), _ld(Z), ids.data_ptr() if ids is not None else 0,
+                                        pos.data_ptr() if pos is not None else 0, n, seq_len, Xh.data_ptr(),
+                                        _ld(Xh), ss.data_ptr(), self.dev_status.data_ptr(), _stream())
+        return Xh, ss
+
     def grad_project(self, G: torch.Tensor, full: bool = False, coeff: bool = True,
                      out: Optional[torch.Tensor] = None, out_full: Optional[torch.Tensor] = None):
         n = G.shape[0]
