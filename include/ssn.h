@@ -404,7 +404,7 @@ enum {
 #define SSN_KVAR_ALT 8    /* MMA_SYNC: 32 rows per warp; EXPAND64: one P row per 16-sequence tile;
                              UMMA_PROJECT: positional product shared per block; UMMA_EXPAND:
                              tiles of 8 sequences x 16 positions; UMMA_ROUNDTRIP: LEFT          */
-#define SSN_KVAR_ROWSUMSQ 16 /* UMMA_EXPAND / EXPAND64 / GENERIC: the row statistic is produced  */
+#define SSN_KVAR_ROWSUMSQ 16 /* UMMA_EXPAND / GENERIC: the row statistic is produced              */
 int32_t ssn_last_kernel(void);
 
 /*

@@ -151,6 +151,83 @@ __host__ __device__ constexpr uint32_t umma_idesc(int n, bool negate_a) {
          ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kUmmaTile >> 4) << 24);
 }
 
+// Last step of the projection epilogue for the token t whose KN accumulator values are in v:
+// subtracts the terms that come from the prepared tables E U and P U (fp32) instead of an operand
+// (sub_eu / sub_pu: that term has no operand in this launch), then stores the row of Z, in the
+// storage dtype or as a wire row of fp32 words followed by the token id.
+template <int KN>
+__device__ __forceinline__ void store_projected_row(const MmaArgs &a, int64_t t, uint32_t (&v)[KN / 16][16],
+                                                    bool sub_eu, bool sub_pu, bool vec) {
+  auto subtract_row = [&](const float *row) {
+    const bool vec4 = (reinterpret_cast<uintptr_t>(row) & 15) == 0;   // 128-bit loads inside the row
+#pragma unroll
+    for (int q = 0; q < KN / 16; ++q)
+#pragma unroll
+      for (int i = 0; i < 16; i += 4) {
+        const int col = q * 16 + i;
+        if (vec4 && col + 4 <= a.k) {
+          const float4 w = __ldg(reinterpret_cast<const float4 *>(row + col));
+          v[q][i] = __float_as_uint(__uint_as_float(v[q][i]) - w.x);
+          v[q][i + 1] = __float_as_uint(__uint_as_float(v[q][i + 1]) - w.y);
+          v[q][i + 2] = __float_as_uint(__uint_as_float(v[q][i + 2]) - w.z);
+          v[q][i + 3] = __float_as_uint(__uint_as_float(v[q][i + 3]) - w.w);
+        } else {
+#pragma unroll
+          for (int e = 0; e < 4; ++e)
+            if (col + e < a.k)
+              v[q][i + e] = __float_as_uint(__uint_as_float(v[q][i + e]) - __ldg(row + col + e));
+        }
+      }
+  };
+  if (sub_eu && a.shift.EU != nullptr) {
+    const int64_t er = embedding_row(a.shift, t);
+    if (er >= 0) subtract_row(a.shift.EU + er * a.shift.ldeu);
+  }
+  if (sub_pu && a.shift.PU != nullptr) {
+    const int64_t pr = position_row(a.shift, t);
+    if (pr >= 0) subtract_row(a.shift.PU + pr * a.shift.ldpu);
+  }
+  if (a.zout32 != nullptr) {   // wire row: fp32 coordinates, then the token id
+    float *wrow = a.zout32 + t * a.ldzout32;
+    const bool vec4 = ((a.ldzout32 & 3) == 0) && ((reinterpret_cast<uintptr_t>(a.zout32) & 15) == 0);
+#pragma unroll
+    for (int q = 0; q < KN / 16; ++q)
+#pragma unroll
+      for (int i = 0; i < 16; i += 4) {
+        const int col = q * 16 + i;
+        if (vec4 && col + 4 <= a.k) {
+          *reinterpret_cast<uint4 *>(wrow + col) = make_uint4(v[q][i], v[q][i + 1], v[q][i + 2], v[q][i + 3]);
+        } else {
+#pragma unroll
+          for (int e = 0; e < 4; ++e)
+            if (col + e < a.k) wrow[col + e] = __uint_as_float(v[q][i + e]);
+        }
+      }
+    if (a.wire_ids != nullptr) reinterpret_cast<int32_t *>(wrow)[a.k] = a.wire_ids[t];
+    return;
+  }
+  __nv_bfloat16 *zrow = a.zout + t * a.ldzout;
+#pragma unroll
+  for (int q = 0; q < KN / 16; ++q) {
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      const int col = q * 16 + h * 8;
+      if (vec && col + 8 <= a.k) {
+        uint4 o;
+        o.x = pack_bf16(__uint_as_float(v[q][h * 8 + 0]), __uint_as_float(v[q][h * 8 + 1]));
+        o.y = pack_bf16(__uint_as_float(v[q][h * 8 + 2]), __uint_as_float(v[q][h * 8 + 3]));
+        o.z = pack_bf16(__uint_as_float(v[q][h * 8 + 4]), __uint_as_float(v[q][h * 8 + 5]));
+        o.w = pack_bf16(__uint_as_float(v[q][h * 8 + 6]), __uint_as_float(v[q][h * 8 + 7]));
+        *reinterpret_cast<uint4 *>(zrow + col) = o;
+      } else {
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+          if (col + i < a.k) zrow[col + i] = __float2bfloat16_rn(__uint_as_float(v[q][h * 8 + i]));
+      }
+    }
+  }
+}
+
 template <int NTP, bool HAS_E, bool HAS_P>
 struct UmmaProjectConfig {
   static_assert(NTP % 2 == 0 && NTP >= 2 && NTP <= 16, "N = 8*NTP must be a multiple of 16 up to 128");
@@ -189,6 +266,39 @@ struct UmmaProjectConfig {
 struct UmmaMaps {
   CUtensorMap x, p, u, u_wide, x2;
 };
+
+// Launches `kernel(a, maps)` as pairs of CTAs (clusters of two) that share their odd tile, one
+// pair per two SMs; falls back to single CTAs where clusters cannot be scheduled.
+template <typename Kernel>
+cudaError_t launch_tile_pairs(Kernel kernel, int threads, int smem, const MmaArgs &a, const UmmaMaps &maps,
+                              int sm_count, cudaStream_t stream) {
+  const int64_t ntiles = (a.n + kUmmaTile - 1) / kUmmaTile;
+  int64_t pairs = ntiles;   // with few tiles every pair has one and splits it over d
+  if (pairs > sm_count / 2) pairs = sm_count / 2;
+  if (pairs < 1) {   // a single SM: plain launch
+    kernel<<<(unsigned)(ntiles < sm_count ? ntiles : sm_count), threads, smem, stream>>>(a, maps);
+    return cudaGetLastError();
+  }
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)(2 * pairs));
+  cfg.blockDim = dim3((unsigned)threads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, a, maps);
+  if (e == cudaSuccess) return e;
+  // a device that cannot co-schedule the pairs: the same kernel without clusters
+  cudaGetLastError();
+  const int64_t grid = ntiles < sm_count ? ntiles : sm_count;
+  kernel<<<(unsigned)grid, threads, smem, stream>>>(a, maps);
+  return cudaGetLastError();
+}
 
 template <int NTP, bool HAS_E, bool HAS_P>
 __global__ void __launch_bounds__(kUmmaThreads, 1)
@@ -532,75 +642,7 @@ codec_umma_project_kernel(const MmaArgs a, const __grid_constant__ UmmaMaps maps
 
       const int64_t t = tile * kUmmaTile + quarter * 32 + lane;
       if (t < a.n) {
-        // terms that come from the prepared tables E U and P U (fp32) instead of an operand
-        auto subtract_row = [&](const float *row) {
-          const bool vec4 = (reinterpret_cast<uintptr_t>(row) & 15) == 0;   // 128-bit loads inside the row
-#pragma unroll
-          for (int q = 0; q < Cfg::kN / 16; ++q)
-#pragma unroll
-            for (int i = 0; i < 16; i += 4) {
-              const int col = q * 16 + i;
-              if (vec4 && col + 4 <= a.k) {
-                const float4 w = __ldg(reinterpret_cast<const float4 *>(row + col));
-                v[q][i] = __float_as_uint(__uint_as_float(v[q][i]) - w.x);
-                v[q][i + 1] = __float_as_uint(__uint_as_float(v[q][i + 1]) - w.y);
-                v[q][i + 2] = __float_as_uint(__uint_as_float(v[q][i + 2]) - w.z);
-                v[q][i + 3] = __float_as_uint(__uint_as_float(v[q][i + 3]) - w.w);
-              } else {
-#pragma unroll
-                for (int e = 0; e < 4; ++e)
-                  if (col + e < a.k)
-                    v[q][i + e] = __float_as_uint(__uint_as_float(v[q][i + e]) - __ldg(row + col + e));
-              }
-            }
-        };
-        if (!HAS_E && a.shift.EU != nullptr) {
-          const int64_t er = embedding_row(a.shift, t);
-          if (er >= 0) subtract_row(a.shift.EU + er * a.shift.ldeu);
-        }
-        if (!HAS_P && a.shift.PU != nullptr) {
-          const int64_t pr = position_row(a.shift, t);
-          if (pr >= 0) subtract_row(a.shift.PU + pr * a.shift.ldpu);
-        }
-        if (a.zout32 != nullptr) {   // wire row: fp32 coordinates, then the token id
-          float *wrow = a.zout32 + t * a.ldzout32;
-          const bool vec4 = ((a.ldzout32 & 3) == 0) && ((reinterpret_cast<uintptr_t>(a.zout32) & 15) == 0);
-#pragma unroll
-          for (int q = 0; q < Cfg::kN / 16; ++q)
-#pragma unroll
-            for (int i = 0; i < 16; i += 4) {
-              const int col = q * 16 + i;
-              if (vec4 && col + 4 <= a.k) {
-                *reinterpret_cast<uint4 *>(wrow + col) = make_uint4(v[q][i], v[q][i + 1], v[q][i + 2], v[q][i + 3]);
-              } else {
-#pragma unroll
-                for (int e = 0; e < 4; ++e)
-                  if (col + e < a.k) wrow[col + e] = __uint_as_float(v[q][i + e]);
-              }
-            }
-          if (a.wire_ids != nullptr) reinterpret_cast<int32_t *>(wrow)[a.k] = a.wire_ids[t];
-          continue;
-        }
-        __nv_bfloat16 *zrow = a.zout + t * a.ldzout;
-#pragma unroll
-        for (int q = 0; q < Cfg::kN / 16; ++q) {
-#pragma unroll
-          for (int h = 0; h < 2; ++h) {
-            const int col = q * 16 + h * 8;
-            if (vec && col + 8 <= a.k) {
-              uint4 o;
-              o.x = pack_bf16(__uint_as_float(v[q][h * 8 + 0]), __uint_as_float(v[q][h * 8 + 1]));
-              o.y = pack_bf16(__uint_as_float(v[q][h * 8 + 2]), __uint_as_float(v[q][h * 8 + 3]));
-              o.z = pack_bf16(__uint_as_float(v[q][h * 8 + 4]), __uint_as_float(v[q][h * 8 + 5]));
-              o.w = pack_bf16(__uint_as_float(v[q][h * 8 + 6]), __uint_as_float(v[q][h * 8 + 7]));
-              *reinterpret_cast<uint4 *>(zrow + col) = o;
-            } else {
-#pragma unroll
-              for (int i = 0; i < 8; ++i)
-                if (col + i < a.k) zrow[col + i] = __float2bfloat16_rn(__uint_as_float(v[q][h * 8 + i]));
-            }
-          }
-        }
+        store_projected_row<Cfg::kN>(a, t, v, !HAS_E, !HAS_P, vec);
       }
     }
   }

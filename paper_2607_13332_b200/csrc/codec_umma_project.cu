@@ -17,33 +17,7 @@ cudaError_t launch_umma_one(const MmaArgs &a, const UmmaMaps &maps, int sm_count
   }
   note_kernel(SSN_KERNEL_UMMA_PROJECT, (HAS_E ? SSN_KVAR_E : 0) | (HAS_P ? SSN_KVAR_P : 0) |
                                            (NTP > 8 ? SSN_KVAR_WIDE : 0) | (a.pshare ? SSN_KVAR_ALT : 0));
-  // pairs of CTAs (clusters of two) that share their odd tile; see the kernel's schedule
-  const int64_t ntiles = (a.n + kUmmaTile - 1) / kUmmaTile;
-  int64_t pairs = ntiles;   // with few tiles every pair has one and splits it over d
-  if (pairs > sm_count / 2) pairs = sm_count / 2;
-  if (pairs < 1) {   // a single SM: plain launch
-    kernel<<<(unsigned)(ntiles < sm_count ? ntiles : sm_count), kUmmaThreads, smem, stream>>>(a, maps);
-    return cudaGetLastError();
-  }
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)(2 * pairs));
-  cfg.blockDim = dim3(kUmmaThreads);
-  cfg.dynamicSmemBytes = smem;
-  cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = 2;
-  attr[0].val.clusterDim.y = 1;
-  attr[0].val.clusterDim.z = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, a, maps);
-  if (e == cudaSuccess) return e;
-  // a device that cannot co-schedule the pairs: the same kernel without clusters
-  cudaGetLastError();
-  const int64_t grid = ntiles < sm_count ? ntiles : sm_count;
-  kernel<<<(unsigned)grid, kUmmaThreads, smem, stream>>>(a, maps);
-  return cudaGetLastError();
+  return launch_tile_pairs(kernel, kUmmaThreads, smem, a, maps, sm_count, stream);
 }
 
 template <int NTP>
