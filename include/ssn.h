@@ -168,8 +168,8 @@ ssn_status_t ssn_decompress(const ssn_codec_t *codec, const void *Z, int64_t ldz
  *             bits may differ from run to run.
  * Everything else as for ssn_decompress.  Performance note: the tensor-core expansion kernel
  * produces the statistic for bf16 codecs with d a multiple of 128, k <= 128, at least 512
- * tokens and, when the codec has P, implicit positions over groups of 8 whole sequences whose
- * length is a multiple of 16; other calls run the general kernel.
+ * tokens and, when the codec has P, implicit positions over whole sequences that tile into g
+ * sequences x 128/g positions (g = 8, or 4, 2, 1 with k <= 64); other calls run the general kernel.
  */
 ssn_status_t ssn_decompress_rowsumsq(const ssn_codec_t *codec, const void *Z, int64_t ldz,
                                      const int32_t *ids, const int32_t *pos, int64_t n_tokens,
@@ -405,6 +405,7 @@ enum {
                              UMMA_PROJECT: positional product shared per block; UMMA_EXPAND:
                              tiles of 8 sequences x 16 positions; UMMA_ROUNDTRIP: LEFT          */
 #define SSN_KVAR_ROWSUMSQ 16 /* UMMA_EXPAND / GENERIC: the row statistic is produced              */
+#define SSN_KVAR_FEWSEQ 32   /* UMMA_EXPAND: tiles of 4, 2 or 1 sequences (a batch that is not groups of 8) */
 int32_t ssn_last_kernel(void);
 
 /*

@@ -7,11 +7,14 @@
 //     D += Sel[128 x 16]   * P_rows[16 x 128]            one MMA, see below
 // and the epilogue adds the gathered E rows in fp32 before the single rounding to bf16.
 //
-// Positions.  With implicit positions (t mod seq_len) a tile is laid out as 8 sequences x 16
-// consecutive positions (a 3-D TMA box), so it needs only 16 rows of P, which enter the
-// accumulator through a constant 0/1 selection matrix (row r selects position r mod 16):
-// 1.0 * bf16 is exact and the sum is taken in fp32, so P costs one MMA per chunk and no thread
-// touches it.  Without P a tile is 128 consecutive tokens.
+// Positions.  With implicit positions (t mod seq_len) a tile is laid out as g sequences x 128/g
+// consecutive positions (a 3-D TMA box), so it needs only 128/g rows of P, which enter the
+// accumulator through a constant 0/1 selection matrix (row r selects position r mod 128/g):
+// 1.0 * bf16 is exact and the sum is taken in fp32, so no thread touches P.  Batches of groups of
+// 8 sequences take g = 8: 16 rows of P and ONE more MMA per chunk (PROWS = 16).  Other batches
+// (the 1 to 6 sequences of a small call) take g = 4, 2 or 1 in the PROWS = 128 variant, which
+// reserves shared memory for up to 128 rows of P per chunk and issues 128/(16 g) MMAs for them.
+// Without P a tile is 128 consecutive tokens.
 //
 //   warp 0     producer: per tile the Z tile; per chunk the 128 rows of U (K-major operand)
 //              and the 16 rows of P.
@@ -36,7 +39,7 @@ namespace ssn {
 
 constexpr int kExpandThreads = 448;
 constexpr int kGatherWarps = 4;
-constexpr int kGridSeqs = 8, kGridPos = 16;   // tile shape with implicit positions
+constexpr int kGridSeqs = 8, kGridPos = 16;   // tile shape of the PROWS = 16 variant
 
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, uint32_t bar,
                                             int c0, int c1, int c2) {
@@ -61,8 +64,9 @@ __device__ __forceinline__ void tma_store_3d(const CUtensorMap *map, uint32_t sr
                ::"l"(map), "r"(src), "r"(c0), "r"(c1), "r"(c2) : "memory");
 }
 
-template <int KG, bool HAS_E, bool HAS_P>
+template <int KG, bool HAS_E, bool HAS_P, int PROWS = kGridPos>
 struct UmmaExpandConfig {
+  static_assert(PROWS == 16 || PROWS == 128, "rows of P per chunk the kernel reserves room for");
   static constexpr int kTileBytes = kUmmaTile * 128;            // [128 rows x 128 B]
   static constexpr int kZBytes = KG * kTileBytes;               // one Z tile: KG groups of 64 coordinates
   // With E and two coordinate groups the E ring would have 4 stages only: one Z tile instead of two
@@ -70,15 +74,17 @@ struct UmmaExpandConfig {
   // load of the next tile's Z).  With one group the ring is deep enough and the second tile pays.
   static constexpr int kZBufs = (HAS_E && KG == 2) ? 1 : 2;
   static constexpr int kU2Bytes = KG * kChunkCols * 128;        // 128 rows of U, K-major, KG groups
-  static constexpr int kPBytes = HAS_P ? 2 * kGridPos * 128 : 0;   // 16 rows of P, two 64-column groups
+  static constexpr int kPBytes = HAS_P ? 2 * PROWS * 128 : 0;      // PROWS rows of P, two 64-column groups
+  static constexpr int kSelBytes = HAS_P ? (PROWS <= 64 ? 1 : 2) * kTileBytes : 0;   // one tile per 64 positions
   static constexpr int kUStageBytes = kU2Bytes + kPBytes;
-  static constexpr int kUStages = (HAS_E || KG == 2) ? 2 : 3;   // with E the shared memory is better spent on its ring
+  // with E the shared memory is better spent on its ring; 128 rows of P per stage leave room for two
+  static constexpr int kUStages = (HAS_E || KG == 2 || (HAS_P && PROWS > kGridPos)) ? 2 : 3;
   static constexpr int kEStageBytes = kTileBytes;               // E rows of 64 columns of a chunk
   // Without E the epilogue warps stage their output in two [32 x 128 B] slabs each; with E the
   // sum is formed in place in the E stage, which is then the source of the TMA store.
   static constexpr int kStagingBytes = HAS_E ? 0 : 8 * 2 * 4096;
   static constexpr int kFixedBytes =
-      kZBufs * kZBytes + (HAS_P ? kTileBytes : 0) + kUStages * kUStageBytes + kStagingBytes;
+      kZBufs * kZBytes + kSelBytes + kUStages * kUStageBytes + kStagingBytes;
   static constexpr int kMaxSmem = 227 * 1024;
   static constexpr int kEFit = (kMaxSmem - 1024 - 512 - kFixedBytes) / kEStageBytes;
   static constexpr int kEStages = HAS_E ? (kEFit < 12 ? kEFit : 12) : 0;
@@ -87,6 +93,7 @@ struct UmmaExpandConfig {
   static constexpr int SE = HAS_E ? kEStages : 1;
   static constexpr int kBars = 4 + 2 * kUStages + 2 * SE + 4;
   static constexpr int kSmemBytes = 1024 + kFixedBytes + kEStages * kEStageBytes + kBars * 8 + 16;
+  static_assert(kSmemBytes <= kMaxSmem, "the rings do not fit in shared memory");
 };
 
 struct UmmaExpandMaps {
@@ -96,16 +103,19 @@ struct UmmaExpandMaps {
 };
 
 struct ExpandGeometry {
-  int32_t grid_mode;      // 1: tiles of 8 sequences x 16 positions, 0: 128 consecutive tokens
+  int32_t grid_mode;      // 1: tiles of gseqs sequences x gpos positions, 0: 128 consecutive tokens
   int32_t seq_len;
-  int32_t nsg;            // groups of 8 sequences
+  int32_t nsg;            // groups of gseqs sequences
+  int32_t gseqs, gpos;    // gseqs * gpos == 128
   int64_t ntiles;
 };
 
-template <int KG, bool HAS_E, bool HAS_P>
+template <int KG, bool HAS_E, bool HAS_P, int PROWS = kGridPos>
 __global__ void __launch_bounds__(kExpandThreads, 1)
 codec_umma_expand_kernel(const MmaArgs a, const ExpandGeometry geo, const __grid_constant__ UmmaExpandMaps maps) {
-  using Cfg = UmmaExpandConfig<KG, HAS_E, HAS_P>;
+  using Cfg = UmmaExpandConfig<KG, HAS_E, HAS_P, PROWS>;
+  // positions and sequences of a tile: fixed in the PROWS = 16 variant, the launch's otherwise
+  const int gpos = PROWS == kGridPos ? kGridPos : geo.gpos, gseqs = PROWS == kGridPos ? kGridSeqs : geo.gseqs;
   constexpr int SU = Cfg::kUStages, SE = Cfg::SE;
   extern __shared__ __align__(128) unsigned char smem_raw[];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -116,7 +126,7 @@ codec_umma_expand_kernel(const MmaArgs a, const ExpandGeometry geo, const __grid
   const uint32_t smem0 = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t z_base = smem0;                                         // the Z tiles
   const uint32_t sel = z_base + Cfg::kZBufs * Cfg::kZBytes;              // selection matrix (HAS_P)
-  const uint32_t u_ring = sel + (HAS_P ? Cfg::kTileBytes : 0);
+  const uint32_t u_ring = sel + Cfg::kSelBytes;
   const uint32_t staging = u_ring + SU * Cfg::kUStageBytes;
   const uint32_t e_ring = staging + Cfg::kStagingBytes;
   const uint32_t bars = e_ring + Cfg::kEStages * Cfg::kEStageBytes;
@@ -133,19 +143,21 @@ codec_umma_expand_kernel(const MmaArgs a, const ExpandGeometry geo, const __grid
       reinterpret_cast<volatile uint32_t *>(smem_raw + (tmem_slot - smem_u32(smem_raw)));
 
   if (HAS_P) {
-    // Sel[r][j] = 1 for j == r mod 16 (K-major, 128-byte rows, swizzled); only K = 16 is read
-    for (uint32_t i = threadIdx.x; i < Cfg::kTileBytes / 16; i += blockDim.x) {
-      const uint32_t r = i >> 3, c = i & 7;     // row, logical 16-byte piece
+    // Sel[r][j] = 1 for j == r mod gpos (K-major, 128-byte rows of 64 positions, swizzled; a second
+    // tile holds positions 64..127); only K = gpos is read
+    for (uint32_t i = threadIdx.x; i < Cfg::kSelBytes / 16; i += blockDim.x) {
+      const uint32_t tile = i / (Cfg::kTileBytes / 16), ii = i % (Cfg::kTileBytes / 16);
+      const uint32_t r = ii >> 3, c = ii & 7;     // row, logical 16-byte piece
       uint4 v = make_uint4(0, 0, 0, 0);
-      const uint32_t j = r & 15;
-      if (c == (j >> 3)) {
+      const uint32_t j = r % (uint32_t)gpos;      // the position row r selects
+      if (tile == (j >> 6) && c == ((j & 63) >> 3)) {
         const uint32_t e = j & 7, word = 0x3F80u << ((e & 1) * 16);
         if ((e >> 1) == 0) v.x = word;
         if ((e >> 1) == 1) v.y = word;
         if ((e >> 1) == 2) v.z = word;
         if ((e >> 1) == 3) v.w = word;
       }
-      const uint32_t off = r * 128 + ((c ^ (r & 7)) << 4);
+      const uint32_t off = tile * Cfg::kTileBytes + r * 128 + ((c ^ (r & 7)) << 4);
       *reinterpret_cast<uint4 *>(smem_raw + (sel - smem_u32(smem_raw)) + off) = v;
     }
     asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
@@ -194,8 +206,8 @@ codec_umma_expand_kernel(const MmaArgs a, const ExpandGeometry geo, const __grid
   auto tile_coords = [&](int64_t tile, int &c1, int &c2) {
     if (geo.grid_mode) {
       const int64_t pb = tile / geo.nsg;
-      c1 = (int)pb * kGridPos;
-      c2 = (int)(tile - pb * geo.nsg) * kGridSeqs;
+      c1 = (int)pb * gpos;
+      c2 = (int)(tile - pb * geo.nsg) * gseqs;
     } else {
       c1 = (int)(tile * kUmmaTile);
       c2 = 0;
@@ -228,7 +240,7 @@ codec_umma_expand_kernel(const MmaArgs a, const ExpandGeometry geo, const __grid
         if (!dead && !mbar_wait(u_empty_bar(slot), parity)) timed_out();
         const uint32_t base = u_ring + (uint32_t)slot * Cfg::kUStageBytes;
         if (lane == 0) {
-          mbar_expect_tx(u_full_bar(slot), Cfg::kUStageBytes);
+          mbar_expect_tx(u_full_bar(slot), Cfg::kU2Bytes + (HAS_P ? 2 * gpos * 128 : 0));
 #pragma unroll
           for (int kg = 0; kg < KG; ++kg) {   // per group of 64 coordinates: 128 rows of 128 bytes
             tma_load_2d(base + kg * Cfg::kTileBytes, &maps.u_wide, u_full_bar(slot), kg * 64, q * kChunkCols);
@@ -254,7 +266,7 @@ codec_umma_expand_kernel(const MmaArgs a, const ExpandGeometry geo, const __grid
       constexpr uint32_t idesc_kk = umma_idesc_kk(kChunkCols);            // Z tile x U chunk, both K-major
       constexpr uint32_t idesc_kmn = umma_idesc(kChunkCols, false);       // Sel (K-major) x P rows (MN-major)
       const uint64_t kdesc = umma_desc(0, 16, 1024, 2);
-      const uint64_t pdesc = umma_desc(0, kGridPos * 128, 1024, 2);       // 64-column groups 2048 bytes apart
+      const uint64_t pdesc = umma_desc(0, (uint32_t)gpos * 128, 1024, 2); // 64-column groups gpos rows apart
       const uint64_t seld = kdesc + umma_desc_addr(sel);
       int slot = 0;
       uint32_t parity = 0;
@@ -277,7 +289,14 @@ codec_umma_expand_kernel(const MmaArgs a, const ExpandGeometry geo, const __grid
             const uint32_t ko = (uint32_t)(j >> 2) * (Cfg::kTileBytes >> 4) + (uint32_t)(j & 3) * 2;
             umma_bf16(dacc, zd + ko, bd + ko, idesc_kk, j > 0 ? 1u : 0u);
           }
-          if (HAS_P) umma_bf16(dacc, seld, pdesc + umma_desc_addr(base + Cfg::kU2Bytes), idesc_kmn, 1u);
+          if (HAS_P) {
+            // K step j: 16 positions = 32 bytes of a Sel row (a second tile from position 64 on)
+            // and 16 rows = 2048 bytes of the P operand
+            const uint64_t pd = pdesc + umma_desc_addr(base + Cfg::kU2Bytes);
+            for (int j = 0; j < gpos / 16; ++j)
+              umma_bf16(dacc, seld + (uint32_t)(j >> 2) * (Cfg::kTileBytes >> 4) + (uint32_t)(j & 3) * 2,
+                        pd + (uint32_t)j * 128, idesc_kmn, 1u);
+          }
           umma_commit(u_empty_bar(slot));
           umma_commit(d_full_bar(db));
           if (q == q1 - 1) umma_commit(z_empty_bar(zb));
@@ -306,7 +325,7 @@ codec_umma_expand_kernel(const MmaArgs a, const ExpandGeometry geo, const __grid
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
           const int r = gw * 32 + i * 4 + sub;
-          const int64_t t = geo.grid_mode ? (int64_t)(c2 + r / kGridPos) * geo.seq_len + c1 + r % kGridPos
+          const int64_t t = geo.grid_mode ? (int64_t)(c2 + r / gpos) * geo.seq_len + c1 + r % gpos
                                           : (int64_t)c1 + r;
           const int64_t er = t < a.n ? embedding_row(a.shift, t) : -1;
           src[i] = (er >= 0 ? reinterpret_cast<const unsigned char *>(
@@ -344,12 +363,13 @@ codec_umma_expand_kernel(const MmaArgs a, const ExpandGeometry geo, const __grid
       int c1, c2;
       tile_coords(tile, c1, c2);
       // first token row of this warp's 32 rows, as TMA store coordinates
-      const int s1 = geo.grid_mode ? c1 : c1 + quarter * 32;
-      const int s2 = geo.grid_mode ? c2 + quarter * (32 / kGridPos) : 0;
+      // (32 rows are 32 / gpos whole sequences, or 32 positions of one sequence when gpos >= 32)
+      const int s1 = geo.grid_mode ? c1 + (quarter * 32) % gpos : c1 + quarter * 32;
+      const int s2 = geo.grid_mode ? c2 + (quarter * 32) / gpos : 0;
       const bool rows_live = geo.grid_mode || (int64_t)s1 < a.n;
       // this thread's token (row quarter * 32 + lane of the tile), for the row statistic
       const int trow = quarter * 32 + lane;
-      const int64_t tok = geo.grid_mode ? (int64_t)(c2 + trow / kGridPos) * geo.seq_len + c1 + trow % kGridPos
+      const int64_t tok = geo.grid_mode ? (int64_t)(c2 + trow / gpos) * geo.seq_len + c1 + trow % gpos
                                         : (int64_t)c1 + trow;
       int q0, q1;
       chunk_range(tile, q0, q1);

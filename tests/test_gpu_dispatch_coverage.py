@@ -85,12 +85,37 @@ def test_decompress_tcgen05_ragged_last_tile(k, tables):
     assert codec.take_status() == 0
 
 
+@pytest.mark.parametrize("batch,seq_len", [(161, 128), (1, 2560), (2, 1280), (3, 1024), (4, 640), (6, 512), (12, 1728),
+                                           (166, 128)])
+@pytest.mark.parametrize("tables,k", [("EP", 40), ("P", 64), ("EP", 8)])
+def test_decompress_tcgen05_few_sequences(batch, seq_len, tables, k):
+    """Batches that are not groups of 8 sequences (the 1 to 6 sequences of a small call): tiles of
+    4, 2 or 1 sequences x 32, 64 or 128 positions, whose P rows enter through a wider selection
+    matrix.  From 2560 tokens (below the large-batch limit) to 21248."""
+    # below the large-batch limit the dispatch takes the tcgen05 expansion for wide models only
+    d = 256 if batch > 100 else (1024 if batch * seq_len > LARGE else 2048)
+    wl = synth.Workload("few", d, k, 500, batch, seq_len, synth.BF16, "zipf")
+    t = synth.codec_inputs(wl, seed=batch + k, noise_std=1e-3)
+    dt, n = wl.dtype, wl.n_tokens
+    E0 = t["E"] if "E" in tables else None
+    codec = Codec(dt, to_device(t["U"], dt), to_device(E0, dt), to_device(t["P"], dt))
+    ids = torch.from_numpy(t["ids"]).cuda()
+    out, buf = padded(n, d, d + 64, dt)
+    codec.decompress(to_device(t["Z0"], dt), ids, seq_len=seq_len, out=out)
+    expect_kernel(B.SSN_KERNEL_UMMA_EXPAND, has=_variant_bits(tables) | B.SSN_KVAR_ALT | B.SSN_KVAR_FEWSEQ)
+    Xo, _ = oracle.decompress(f64(t["Z0"], dt), f64(t["U"], dt), f64(E0, dt), t["ids"], f64(t["P"], dt),
+                              oracle.token_positions(n, seq_len))
+    assert_close(host64(out, dt), Xo, dt, f"decompress {batch} x {seq_len} {tables} k={k}")
+    assert guards_intact(out, buf, dt)
+    assert codec.take_status() == 0
+
+
 # ---- decompress on the mma.sync kernels the tcgen05 expansion hands over to ----------------------
 @pytest.mark.parametrize("case", ["batch_not_8", "ragged_length", "explicit_pos", "d192_dedup", "d192_noshift",
                                   "d160", "d160_wide", "k72_explicit_pos"])
 def test_decompress_mma_sync_large_batches(case):
     batch, seq_len, d, k, tables, explicit = {
-        "batch_not_8": (161, 128, 256, 40, "EP", False),        # batch not a multiple of 8
+        "batch_not_8": (161, 128, 256, 72, "EP", False),        # odd batch and a rank above 64
         "ragged_length": (1, 160 * 128 + 11, 256, 24, "EP", False),   # length not a multiple of 16
         "explicit_pos": (160, 128, 256, 40, "EP", True),        # positions given per token
         "d192_dedup": (160, 128, 192, 40, "EP", False),         # d % 128 != 0, 16-sequence tiles share a P row
@@ -110,7 +135,7 @@ def test_decompress_mma_sync_large_batches(case):
     out, buf = padded(n, d, d + 32, dt)
     codec.decompress(to_device(t["Z0"], dt), ids, seq_len=seq_len, pos=pos, out=out)
     want = {
-        "batch_not_8": (B.SSN_KERNEL_EXPAND64, B.SSN_KVAR_E | B.SSN_KVAR_P, B.SSN_KVAR_ALT),
+        "batch_not_8": (B.SSN_KERNEL_MMA_SYNC, B.SSN_KVAR_E | B.SSN_KVAR_P | B.SSN_KVAR_WIDE, 0),
         "ragged_length": (B.SSN_KERNEL_EXPAND64, B.SSN_KVAR_E | B.SSN_KVAR_P, B.SSN_KVAR_ALT),
         "explicit_pos": (B.SSN_KERNEL_EXPAND64, B.SSN_KVAR_E | B.SSN_KVAR_P, B.SSN_KVAR_ALT),
         "d192_dedup": (B.SSN_KERNEL_EXPAND64, B.SSN_KVAR_E | B.SSN_KVAR_P | B.SSN_KVAR_ALT, 0),

@@ -52,6 +52,12 @@ def test_rowsumsq_on_the_tcgen05_expansion(batch, seq_len, d, k, tables):
     _check(wl, tables, B.SSN_KERNEL_UMMA_EXPAND, ld_pad=64, seed=batch + k)
 
 
+@pytest.mark.parametrize("batch,seq_len", [(2, 2048), (3, 1024), (6, 512)])
+def test_rowsumsq_few_sequences_on_the_tcgen05_expansion(batch, seq_len):
+    wl = synth.Workload("stat", 512, 40, 300, batch, seq_len, synth.BF16, "zipf")
+    _check(wl, "EP", B.SSN_KERNEL_UMMA_EXPAND, ld_pad=8, seed=batch)
+
+
 def test_rowsumsq_ragged_token_count_on_the_tcgen05_expansion():
     wl = synth.Workload("stat", 128, 24, 300, 1, 5 * 128 + 11, synth.BF16, "zipf")
     _check(wl, "E", B.SSN_KERNEL_UMMA_EXPAND, ld_pad=8)
