@@ -1,6 +1,6 @@
 // General kernels of libssn: any element type, any rank, any leading dimension or alignment.
 // They are the fp32 path and the fallback for shapes the tensor-core kernels do not take.
-// Plain fp32 FMAs; one warp owns one token (or one row of W) and reduces over d with shuffles.
+// Plain fp32 FMAs; a warp owns two tokens (or rows of W), U is staged through shared memory.
 #pragma once
 
 #include "ssn_common.cuh"
@@ -32,93 +32,196 @@ struct TokenArgs {
 };
 
 constexpr int kGenericWarps = 8;
-constexpr int kGenericKChunk = 8;
+constexpr int kGenericKChunk = 8;     // coordinates per pass of the table and LEFT kernels below
+constexpr int kGenericTokens = 2;     // tokens per warp
+constexpr int kGenericCoords = 32;    // coordinates per pass
+constexpr int kGenericRows = 64;      // rows of U staged in shared memory at a time (two per lane)
+constexpr int kGenericTokensPerBlock = kGenericWarps * kGenericTokens;
 
+// Dynamic shared memory: the coordinates of the block's tokens (fp32) and one staged piece of U.
+inline size_t generic_token_smem_bytes(int k) {
+  return ((size_t)kGenericTokensPerBlock * k + (size_t)kGenericRows * (kGenericCoords + 1)) * sizeof(float);
+}
+
+// A warp owns kGenericTokens tokens; its lanes split d.  U is staged through shared memory in
+// pieces of kGenericRows rows x kGenericCoords coordinates (fp32, row pitch odd, so that the lanes,
+// which read different rows, hit different banks) by all warps of the block together, and every
+// staged value is used for both tokens of every warp.
+//   projection: lane l holds rows l and l + 32 of the piece: r = x - e - p for both tokens, then
+//       acc[token][coordinate] += r * U[row][coordinate] for the 32 coordinates of the pass;
+//       shuffle reduction over the lanes at the end of a pass.  The row is re-read once per pass.
+//   expansion: lane l produces columns l and l + 32 of the piece: acc[token][column] +=
+//       z[token][coordinate] * U[column][coordinate] over all passes, then the shift terms are
+//       added and the row statistic (if asked for) is summed before the rounding.
 template <typename T>
 __global__ void __launch_bounds__(kGenericWarps * 32)
 token_kernel(const TokenArgs a) {
-  extern __shared__ float zs_all[];
+  extern __shared__ float smem_f[];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int64_t t = (int64_t)blockIdx.x * kGenericWarps + warp;
-  if (t >= a.n) return;
-  float *zs = zs_all + (size_t)warp * a.k;
+  float *zs = smem_f + (size_t)warp * kGenericTokens * a.k;               // [token][k] of this warp
+  float *us = smem_f + (size_t)kGenericTokensPerBlock * a.k;              // [kGenericRows][kGenericCoords + 1]
+  constexpr int kPitch = kGenericCoords + 1;
+  const int64_t t0 = ((int64_t)blockIdx.x * kGenericWarps + warp) * kGenericTokens;
   const T *U = static_cast<const T *>(a.U);
 
-  const T *erow = nullptr, *prow = nullptr;
-  if (a.sub_shift || a.add_shift) {
-    int64_t er = embedding_row(a.shift, t), pr = position_row(a.shift, t);
-    if (er >= 0) erow = static_cast<const T *>(a.shift.E) + er * a.shift.lde;
-    if (pr >= 0) prow = static_cast<const T *>(a.shift.P) + pr * a.shift.ldp;
+  bool valid[kGenericTokens];
+  const T *erow[kGenericTokens], *prow[kGenericTokens];
+#pragma unroll
+  for (int tk = 0; tk < kGenericTokens; ++tk) {
+    valid[tk] = t0 + tk < a.n;
+    erow[tk] = prow[tk] = nullptr;
+    if (valid[tk] && (a.sub_shift || a.add_shift)) {
+      const int64_t er = embedding_row(a.shift, t0 + tk), pr = position_row(a.shift, t0 + tk);
+      if (er >= 0) erow[tk] = static_cast<const T *>(a.shift.E) + er * a.shift.lde;
+      if (pr >= 0) prow[tk] = static_cast<const T *>(a.shift.P) + pr * a.shift.ldp;
+    }
   }
+  // stages rows [i0, i0 + kGenericRows) x coordinates [j0, j0 + kGenericCoords) of `src` (zeros outside)
+  auto stage_u = [&](const T *src, int64_t ld, int rows, int i0, int j0) {
+    __syncthreads();   // the previous piece has been read by everyone
+    for (int e = threadIdx.x; e < kGenericRows * kGenericCoords; e += kGenericWarps * 32) {
+      const int ii = e / kGenericCoords, jj = e % kGenericCoords;
+      const int i = i0 + ii, j = j0 + jj;
+      us[ii * kPitch + jj] = (i < rows && j < a.k) ? to_f32(src[(int64_t)i * ld + j]) : 0.f;
+    }
+    __syncthreads();
+  };
 
   if (a.src != nullptr) {
-    const T *x = static_cast<const T *>(a.src) + t * a.lds;
-    const T *x2 = a.src2 != nullptr ? static_cast<const T *>(a.src2) + t * a.lds2 : nullptr;
-    for (int j0 = 0; j0 < a.k; j0 += kGenericKChunk) {
-      float acc[kGenericKChunk];
+    const T *x[kGenericTokens], *x2[kGenericTokens];
 #pragma unroll
-      for (int jj = 0; jj < kGenericKChunk; ++jj) acc[jj] = 0.f;
-      const int jn = min(kGenericKChunk, a.k - j0);
-      for (int i = lane; i < a.d; i += 32) {
-        float r = to_f32(x[i]);
-        if (x2 != nullptr) r += to_f32(x2[i]);
-        if (a.sub_shift) {
-          if (erow) r -= to_f32(erow[i]);
-          if (prow) r -= to_f32(prow[i]);
+    for (int tk = 0; tk < kGenericTokens; ++tk) {
+      x[tk] = static_cast<const T *>(a.src) + (valid[tk] ? t0 + tk : 0) * a.lds;
+      x2[tk] = a.src2 != nullptr ? static_cast<const T *>(a.src2) + (valid[tk] ? t0 + tk : 0) * a.lds2 : nullptr;
+    }
+    for (int j0 = 0; j0 < a.k; j0 += kGenericCoords) {
+      float acc[kGenericTokens][kGenericCoords];
+#pragma unroll
+      for (int tk = 0; tk < kGenericTokens; ++tk)
+#pragma unroll
+        for (int jj = 0; jj < kGenericCoords; ++jj) acc[tk][jj] = 0.f;
+      for (int i0 = 0; i0 < a.d; i0 += kGenericRows) {
+        // the residuals of this piece first: their loads are in flight while U is being staged
+        float r[kGenericRows / 32][kGenericTokens];
+#pragma unroll
+        for (int h = 0; h < kGenericRows / 32; ++h) {
+          const int i = i0 + lane + 32 * h;
+#pragma unroll
+          for (int tk = 0; tk < kGenericTokens; ++tk) {
+            float v = 0.f;
+            if (valid[tk] && i < a.d) {
+              v = to_f32(x[tk][i]);
+              if (x2[tk] != nullptr) v += to_f32(x2[tk][i]);
+              if (a.sub_shift) {
+                if (erow[tk]) v -= to_f32(erow[tk][i]);
+                if (prow[tk]) v -= to_f32(prow[tk][i]);
+              }
+            }
+            r[h][tk] = v;
+          }
         }
-        const T *urow = U + (int64_t)i * a.ldu + j0;
+        stage_u(U, a.ldu, a.d, i0, j0);
 #pragma unroll
-        for (int jj = 0; jj < kGenericKChunk; ++jj)
-          if (jj < jn) acc[jj] = fmaf(r, to_f32(urow[jj]), acc[jj]);
+        for (int h = 0; h < kGenericRows / 32; ++h) {
+          const float *urow = us + (lane + 32 * h) * kPitch;
+#pragma unroll
+          for (int jj = 0; jj < kGenericCoords; ++jj) {
+            const float u = urow[jj];
+#pragma unroll
+            for (int tk = 0; tk < kGenericTokens; ++tk) acc[tk][jj] = fmaf(r[h][tk], u, acc[tk][jj]);
+          }
+        }
       }
 #pragma unroll
-      for (int jj = 0; jj < kGenericKChunk; ++jj) {
-        float v = acc[jj];
+      for (int tk = 0; tk < kGenericTokens; ++tk)
 #pragma unroll
-        for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
-        if (lane == 0 && jj < jn) zs[j0 + jj] = v;
+        for (int jj = 0; jj < kGenericCoords; ++jj) {
+          float v = acc[tk][jj];
+#pragma unroll
+          for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
+          if (lane == 0 && j0 + jj < a.k) zs[tk * a.k + j0 + jj] = v;
+        }
+    }
+    __syncwarp();
+#pragma unroll
+    for (int tk = 0; tk < kGenericTokens; ++tk) {
+      if (!valid[tk] || a.zout == nullptr) continue;
+      const int64_t t = t0 + tk;
+      if (a.wire) {
+        float *z = static_cast<float *>(a.zout) + t * a.ldzout;
+        for (int j = lane; j < a.k; j += 32) z[j] = zs[tk * a.k + j];
+        if (a.wire_ids && lane == 0) reinterpret_cast<int32_t *>(z)[a.k] = a.shift.ids[t];
+      } else {
+        T *z = static_cast<T *>(a.zout) + t * a.ldzout;
+        for (int j = lane; j < a.k; j += 32) z[j] = from_f32<T>(zs[tk * a.k + j]);
       }
     }
-    __syncwarp();
-    if (a.zout != nullptr && a.wire) {
-      float *z = static_cast<float *>(a.zout) + t * a.ldzout;
-      for (int j = lane; j < a.k; j += 32) z[j] = zs[j];
-      if (a.wire_ids && lane == 0) reinterpret_cast<int32_t *>(z)[a.k] = a.shift.ids[t];
-    } else if (a.zout != nullptr) {
-      T *z = static_cast<T *>(a.zout) + t * a.ldzout;
-      for (int j = lane; j < a.k; j += 32) z[j] = from_f32<T>(zs[j]);
-    }
-  } else if (a.wire) {
-    const float *z = static_cast<const float *>(a.zin) + t * a.ldzin;
-    for (int j = lane; j < a.k; j += 32) zs[j] = z[j];
-    __syncwarp();
   } else {
-    const T *z = static_cast<const T *>(a.zin) + t * a.ldzin;
-    for (int j = lane; j < a.k; j += 32) zs[j] = to_f32(z[j]);
+#pragma unroll
+    for (int tk = 0; tk < kGenericTokens; ++tk) {
+      const int64_t t = valid[tk] ? t0 + tk : 0;
+      if (a.wire) {
+        const float *z = static_cast<const float *>(a.zin) + t * a.ldzin;
+        for (int j = lane; j < a.k; j += 32) zs[tk * a.k + j] = z[j];
+      } else {
+        const T *z = static_cast<const T *>(a.zin) + t * a.ldzin;
+        for (int j = lane; j < a.k; j += 32) zs[tk * a.k + j] = to_f32(z[j]);
+      }
+    }
     __syncwarp();
   }
 
   if (a.dst != nullptr) {
-    T *out = static_cast<T *>(a.dst) + t * a.lddst;
     const T *Ux = a.U2 != nullptr ? static_cast<const T *>(a.U2) : U;
     const int64_t ldux = a.U2 != nullptr ? a.ldu2 : a.ldu;
     const int dx = a.U2 != nullptr ? a.d2 : a.d;
-    float ss = 0.f;
-    for (int i = lane; i < dx; i += 32) {
-      const T *urow = Ux + (int64_t)i * ldux;
-      float acc = 0.f;
-      for (int j = 0; j < a.k; ++j) acc = fmaf(zs[j], to_f32(urow[j]), acc);
-      if (a.add_shift) {
-        if (erow) acc += to_f32(erow[i]);
-        if (prow) acc += to_f32(prow[i]);
+    float ss[kGenericTokens];
+#pragma unroll
+    for (int tk = 0; tk < kGenericTokens; ++tk) ss[tk] = 0.f;
+    for (int i0 = 0; i0 < dx; i0 += kGenericRows) {
+      float acc[kGenericTokens][kGenericRows / 32];
+#pragma unroll
+      for (int tk = 0; tk < kGenericTokens; ++tk)
+#pragma unroll
+        for (int h = 0; h < kGenericRows / 32; ++h) acc[tk][h] = 0.f;
+      for (int j0 = 0; j0 < a.k; j0 += kGenericCoords) {
+        stage_u(Ux, ldux, dx, i0, j0);
+        const int jn = min(kGenericCoords, a.k - j0);
+        for (int jj = 0; jj < jn; ++jj) {
+#pragma unroll
+          for (int h = 0; h < kGenericRows / 32; ++h) {
+            const float u = us[(lane + 32 * h) * kPitch + jj];
+#pragma unroll
+            for (int tk = 0; tk < kGenericTokens; ++tk) acc[tk][h] = fmaf(zs[tk * a.k + j0 + jj], u, acc[tk][h]);
+          }
+        }
       }
-      ss = fmaf(acc, acc, ss);
-      out[i] = from_f32<T>(acc);
+#pragma unroll
+      for (int tk = 0; tk < kGenericTokens; ++tk) {
+        if (!valid[tk]) continue;
+        T *out = static_cast<T *>(a.dst) + (t0 + tk) * a.lddst;
+#pragma unroll
+        for (int h = 0; h < kGenericRows / 32; ++h) {
+          const int i = i0 + lane + 32 * h;
+          if (i >= dx) continue;
+          float v = acc[tk][h];
+          if (a.add_shift) {
+            if (erow[tk]) v += to_f32(erow[tk][i]);
+            if (prow[tk]) v += to_f32(prow[tk][i]);
+          }
+          ss[tk] = fmaf(v, v, ss[tk]);
+          out[i] = from_f32<T>(v);
+        }
+      }
     }
     if (a.rowsumsq != nullptr) {
 #pragma unroll
-      for (int off = 16; off > 0; off >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, off);
-      if (lane == 0) a.rowsumsq[t] = ss;
+      for (int tk = 0; tk < kGenericTokens; ++tk) {
+        float v = ss[tk];
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
+        if (lane == 0 && valid[tk]) a.rowsumsq[t0 + tk] = v;
+      }
     }
   }
 }

@@ -90,20 +90,17 @@ bool mma_eligible(const TokenArgs &a, int32_t dtype) {
 
 ssn_status_t launch_generic_token_kernel(const TokenArgs &a, int32_t dtype, cudaStream_t stream) {
   if (a.n == 0) return SSN_OK;
-  const int64_t blocks = (a.n + kGenericWarps - 1) / kGenericWarps;
+  const int64_t blocks = (a.n + kGenericTokensPerBlock - 1) / kGenericTokensPerBlock;
   if (blocks > 0x7fffffffLL) return SSN_ERR_SHAPE;
-  const size_t smem = (size_t)kGenericWarps * a.k * sizeof(float);
+  const size_t smem = generic_token_smem_bytes(a.k);
+  if (smem > 227 * 1024) return SSN_ERR_SHAPE;   // rank too large for the general kernel's shared memory
   if (smem > 48 * 1024) {
-    cudaError_t e;
-    if (dtype == SSN_F32)
-      e = cudaFuncSetAttribute(token_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                               (int)smem);
-    else
-      e = cudaFuncSetAttribute(token_kernel<__nv_bfloat16>,
-                               cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    static std::atomic<uint64_t> configured_f32{0}, configured_bf16{0};
+    const cudaError_t e = dtype == SSN_F32 ? allow_dynamic_smem(token_kernel<float>, 227 * 1024, configured_f32)
+                                           : allow_dynamic_smem(token_kernel<__nv_bfloat16>, 227 * 1024, configured_bf16);
     if (e != cudaSuccess) {
       cudaGetLastError();
-      return SSN_ERR_SHAPE;  // rank too large for the general kernel's shared memory
+      return SSN_ERR_CUDA;
     }
   }
   if (dtype == SSN_F32)
