@@ -297,9 +297,10 @@ ssn_status_t ssn_head_embed(const ssn_codec_t *codec, const void *Elow, int64_t 
  *                         the rows and the `ids` argument is ignored.  A bf16 codec with
  *                         2 * kpad <= 128 (kpad = k rounded up to 8) runs on the tensor cores
  *                         with the fp32 coordinates split into a bf16 head and a bf16 remainder
- *                         (rank 2 * kpad against the basis repeated twice), which keeps about 16
- *                         of the 24 significand bits of a coordinate, far below the single
- *                         bf16 rounding of X^; for that the call needs a 256-byte aligned workspace of
+ *                         (two products against the same basis, or rank 2 * kpad against the
+ *                         basis repeated twice), which keeps about 16 of the 24 significand bits
+ *                         of a coordinate, far below the single bf16 rounding of X^; for that the
+ *                         call needs a 256-byte aligned workspace of
  *                         ssn_decompress_wire_workspace_bytes() bytes.  With a smaller (or
  *                         misaligned) workspace the general kernel runs; with_ids always needs
  *                         at least n_tokens * 4 bytes (rounded up to 256).
@@ -405,6 +406,7 @@ enum {
                              UMMA_PROJECT: positional product shared per block; UMMA_EXPAND:
                              tiles of 8 sequences x 16 positions; UMMA_ROUNDTRIP: LEFT          */
 #define SSN_KVAR_ROWSUMSQ 16 /* UMMA_EXPAND / GENERIC: the row statistic is produced              */
+#define SSN_KVAR_TWO_RUNS 64  /* UMMA_EXPAND: head and remainder of fp32 wire rows as two runs against one chunk of U */
 #define SSN_KVAR_FEWSEQ 32   /* UMMA_EXPAND: tiles of 4, 2 or 1 sequences (a batch that is not groups of 8) */
 int32_t ssn_last_kernel(void);
 

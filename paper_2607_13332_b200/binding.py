@@ -24,7 +24,7 @@ SSN_DEV_BAD_ID, SSN_DEV_BAD_POS, SSN_DEV_TIMEOUT = 1, 2, 4
 # ssn_last_kernel(): family | variant bits << 8
 (SSN_KERNEL_NONE, SSN_KERNEL_GENERIC, SSN_KERNEL_MMA_SYNC, SSN_KERNEL_MMA_SYNC_DSPLIT, SSN_KERNEL_EXPAND64,
  SSN_KERNEL_UMMA_PROJECT, SSN_KERNEL_UMMA_EXPAND, SSN_KERNEL_UMMA_ROUNDTRIP, SSN_KERNEL_UMMA_TOKENS) = range(9)
-SSN_KVAR_E, SSN_KVAR_P, SSN_KVAR_WIDE, SSN_KVAR_ALT, SSN_KVAR_ROWSUMSQ, SSN_KVAR_FEWSEQ = 1, 2, 4, 8, 16, 32
+SSN_KVAR_E, SSN_KVAR_P, SSN_KVAR_WIDE, SSN_KVAR_ALT, SSN_KVAR_ROWSUMSQ, SSN_KVAR_FEWSEQ, SSN_KVAR_TWO_RUNS = 1, 2, 4, 8, 16, 32, 64
 
 DTYPES = {"f32": SSN_F32, "bf16": SSN_BF16}
 SIDES = {"left": SSN_SIDE_LEFT, "right": SSN_SIDE_RIGHT}

@@ -13,6 +13,9 @@ namespace ssn {
 struct MmaArgs {
   const __nv_bfloat16 *src;   // [n x d] rows to project, or nullptr (expand only)
   const __nv_bfloat16 *zin;   // [n x k] coordinates for expand-only
+  // tcgen05 expansion only, k <= 64: a second [n x k] coordinate matrix (same leading dimension)
+  // whose product with U^T is added to the first one's (the bf16 remainder of fp32 wire rows); nullptr: none
+  const __nv_bfloat16 *zin2;
   __nv_bfloat16 *zout;        // [n x k] coordinates out, nullable
   __nv_bfloat16 *dst;         // [n x d] expansion out, nullable
   const __nv_bfloat16 *U;     // [d x k], 16-byte aligned, ldu % 8 == 0

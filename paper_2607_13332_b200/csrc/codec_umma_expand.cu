@@ -21,7 +21,7 @@ cudaError_t launch_umma_expand_one(const MmaArgs &a, const ExpandGeometry &geo, 
   kernel<<<(unsigned)grid, kExpandThreads, smem, stream>>>(a, geo, maps);
   note_kernel(SSN_KERNEL_UMMA_EXPAND, (HAS_E ? SSN_KVAR_E : 0) | (HAS_P ? SSN_KVAR_P : 0) | (KG == 2 ? SSN_KVAR_WIDE : 0) |
                                           (geo.grid_mode ? SSN_KVAR_ALT : 0) | (a.rowsumsq != nullptr ? SSN_KVAR_ROWSUMSQ : 0) |
-                                          (PROWS != kGridPos ? SSN_KVAR_FEWSEQ : 0));
+                                          (PROWS != kGridPos ? SSN_KVAR_FEWSEQ : 0) | (a.zin2 != nullptr ? SSN_KVAR_TWO_RUNS : 0));
   return cudaGetLastError();
 }
 
@@ -35,6 +35,7 @@ cudaError_t launch_codec_umma_expand(const MmaArgs &a, bool shift, int sm_count,
   if (a.zin == nullptr || a.dst == nullptr || a.src != nullptr) return cudaErrorNotSupported;
   if (a.d % kChunkCols != 0 || a.k > 128 || a.n < 4 * kUmmaTile || a.n > 0x7fffffffLL)
     return cudaErrorNotSupported;
+  if (a.zin2 != nullptr && a.k > 64) return cudaErrorNotSupported;   // two runs share one 64-coordinate U chunk
   const bool has_e = shift && a.shift.E != nullptr, has_p = shift && a.shift.P != nullptr;
   ExpandGeometry geo{};
   geo.seq_len = a.shift.seq_len;
@@ -65,6 +66,10 @@ cudaError_t launch_codec_umma_expand(const MmaArgs &a, bool shift, int sm_count,
     const int out_pos = geo.gpos < 32 ? geo.gpos : 32;
     if (!make_sw128_map3(&maps.z, a.zin, a.k, L, B, a.ldzin, L * a.ldzin, geo.gpos, geo.gseqs))
       return cudaErrorNotSupported;
+    maps.z2 = maps.z;
+    if (a.zin2 != nullptr &&
+        !make_sw128_map3(&maps.z2, a.zin2, a.k, L, B, a.ldzin, L * a.ldzin, geo.gpos, geo.gseqs))
+      return cudaErrorNotSupported;
     if (!make_sw128_map3(&maps.out, a.dst, a.d, L, B, a.lddst, L * a.lddst, out_pos, 32 / out_pos))
       return cudaErrorNotSupported;
     // P as [column group of 64][position][64 columns]: one box of 64 x gpos x 2 is a chunk's rows
@@ -73,6 +78,9 @@ cudaError_t launch_codec_umma_expand(const MmaArgs &a, bool shift, int sm_count,
       return cudaErrorNotSupported;
   } else {
     if (!make_sw128_map3(&maps.z, a.zin, a.k, a.n, 1, a.ldzin, a.n * a.ldzin, kUmmaTile, 1))
+      return cudaErrorNotSupported;
+    maps.z2 = maps.z;
+    if (a.zin2 != nullptr && !make_sw128_map3(&maps.z2, a.zin2, a.k, a.n, 1, a.ldzin, a.n * a.ldzin, kUmmaTile, 1))
       return cudaErrorNotSupported;
     if (!make_sw128_map3(&maps.out, a.dst, a.d, a.n, 1, a.lddst, a.n * a.lddst, 32, 1))
       return cudaErrorNotSupported;

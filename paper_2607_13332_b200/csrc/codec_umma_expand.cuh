@@ -97,6 +97,8 @@ struct UmmaExpandConfig {
 };
 
 struct UmmaExpandMaps {
+  // z2: the second coordinate matrix of a two-run expansion (MmaArgs::zin2), else a copy of z
+  CUtensorMap z2;
   // z: Z tile (box 64 x 128 rows, or 64 x 16 x 8); u / u_wide: 64 x 64 boxes of U (see UmmaMaps);
   // p: P viewed as [column group][row][64 columns], boxes of 64 x 16 rows x 2 groups; out: 64 columns x 32 rows (or 64 x 16 x 2)
   CUtensorMap z, u, u_wide, p, out;
@@ -122,6 +124,10 @@ codec_umma_expand_kernel(const MmaArgs a, const ExpandGeometry geo, const __grid
   const int nchunks = a.d / kChunkCols;
   const int ksteps = (a.k + 15) / 16;
   const int64_t ntiles = geo.ntiles;
+  // Two coordinate matrices (head and remainder of fp32 wire rows) against the same U chunk: both
+  // Z buffers hold one tile's pair, so the tiles are not double-buffered then (KG == 1 only).
+  const bool two_runs = KG == 1 && a.zin2 != nullptr;
+  const int zbufs = two_runs ? 1 : Cfg::kZBufs;
 
   const uint32_t smem0 = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t z_base = smem0;                                         // the Z tiles
@@ -226,13 +232,14 @@ codec_umma_expand_kernel(const MmaArgs a, const ExpandGeometry geo, const __grid
     for (int64_t tile = tile_lo; tile <= tile_hi; ++tile, ++tcount) {
       int c1, c2;
       tile_coords(tile, c1, c2);
-      const int zb = (int)(tcount % Cfg::kZBufs);
-      if (!dead && !mbar_wait(z_empty_bar(zb), (uint32_t)(((tcount / Cfg::kZBufs) & 1) ^ 1))) timed_out();
+      const int zb = (int)(tcount % zbufs);
+      if (!dead && !mbar_wait(z_empty_bar(zb), (uint32_t)(((tcount / zbufs) & 1) ^ 1))) timed_out();
       if (lane == 0) {
-        mbar_expect_tx(z_full_bar(zb), Cfg::kZBytes);
+        mbar_expect_tx(z_full_bar(zb), two_runs ? 2 * Cfg::kTileBytes : Cfg::kZBytes);
 #pragma unroll
         for (int kg = 0; kg < KG; ++kg)
           tma_load_3d(z_base + zb * Cfg::kZBytes + kg * Cfg::kTileBytes, &maps.z, z_full_bar(zb), kg * 64, c1, c2);
+        if (two_runs) tma_load_3d(z_base + Cfg::kTileBytes, &maps.z2, z_full_bar(zb), 0, c1, c2);
       }
       int q0, q1;
       chunk_range(tile, q0, q1);
@@ -272,9 +279,10 @@ codec_umma_expand_kernel(const MmaArgs a, const ExpandGeometry geo, const __grid
       uint32_t parity = 0;
       int64_t tcount = 0, ccount = 0;
       for (int64_t tile = tile_lo; tile <= tile_hi; ++tile, ++tcount) {
-        const int zb = (int)(tcount % Cfg::kZBufs);
-        if (!dead && !mbar_wait(z_full_bar(zb), (uint32_t)((tcount / Cfg::kZBufs) & 1))) timed_out();
+        const int zb = (int)(tcount % zbufs);
+        if (!dead && !mbar_wait(z_full_bar(zb), (uint32_t)((tcount / zbufs) & 1))) timed_out();
         const uint64_t zd = kdesc + umma_desc_addr(z_base + zb * Cfg::kZBytes);
+        const uint64_t zd2 = kdesc + umma_desc_addr(z_base + Cfg::kTileBytes);
         int q0, q1;
         chunk_range(tile, q0, q1);
         for (int q = q0; q < q1; ++q, ++ccount) {
@@ -289,6 +297,8 @@ codec_umma_expand_kernel(const MmaArgs a, const ExpandGeometry geo, const __grid
             const uint32_t ko = (uint32_t)(j >> 2) * (Cfg::kTileBytes >> 4) + (uint32_t)(j & 3) * 2;
             umma_bf16(dacc, zd + ko, bd + ko, idesc_kk, j > 0 ? 1u : 0u);
           }
+          if (two_runs)
+            for (int j = 0; j < ksteps; ++j) umma_bf16(dacc, zd2 + (uint32_t)j * 2, bd + (uint32_t)j * 2, idesc_kk, 1u);
           if (HAS_P) {
             // K step j: 16 positions = 32 bytes of a Sel row (a second tile from position 64 on)
             // and 16 rows = 2048 bytes of the P operand

@@ -638,6 +638,32 @@ ssn_status_t ssn_decompress_wire(const ssn_codec_t *codec, const void *wire, int
     st = launch_status();
     if (st != SSN_OK) return st;
     if (split) {
+      // First choice: the tcgen05 expansion with the head and the remainder as two runs against
+      // the same chunk of U (rank k, the basis as it is).  It refuses what it does not take.
+      const int sms = sm_count_of_current_device();
+      const auto ok16 = [](const void *p, int64_t ld) { return p == nullptr || (aligned16(p) && (ld & 7) == 0); };
+      if (sms > 0 && codec->k <= 64 && ok16(codec->U, codec->ldu) && ok16(Xhat, ldx) && ok16(codec->E, codec->lde) &&
+          ok16(codec->P, codec->ldp)) {
+        MmaArgs m{};
+        m.zin = w.split;
+        m.zin2 = w.split + kp;
+        m.ldzin = 2 * kp;
+        m.dst = static_cast<__nv_bfloat16 *>(Xhat);
+        m.lddst = ldx;
+        m.U = static_cast<const __nv_bfloat16 *>(codec->U);
+        m.ldu = codec->ldu;
+        m.n = n_tokens;
+        m.d = codec->d;
+        m.k = codec->k;
+        m.shift = a.shift;
+        const cudaError_t e = launch_codec_umma_expand(m, a.shift.E != nullptr || a.shift.P != nullptr, sms, s);
+        if (e == cudaSuccess) return launch_status();
+        if (e != cudaErrorNotSupported) {
+          cudaGetLastError();
+          return SSN_ERR_CUDA;
+        }
+      }
+      // otherwise rank 2 kp on whichever kernel takes it: (head | rem)(U | U)^T = (head + rem) U^T
       a.zin = w.split;
       a.ldzin = 2 * kp;
       a.U = w.U2;

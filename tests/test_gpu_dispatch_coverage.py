@@ -192,7 +192,8 @@ def test_compress_tcgen05_large_batches(tables):
 # ---- wire rows and the head-stage input above the limit -------------------------------------------
 @pytest.mark.parametrize("k,with_ids", [(40, True), (40, False), (24, True), (24, False)])
 def test_decompress_wire_large_batches(k, with_ids):
-    """k = 40 expands at rank 80 (two coordinate groups), k = 24 at rank 48 (one)."""
+    """The fp32 coordinates travel as a bf16 head and a bf16 remainder, two products against the
+    same chunk of U on the tcgen05 expansion."""
     wl, t, E0, P0 = _inputs(160, 128, 256, k, 700, seed=k + with_ids, tables="EP")
     dt, n = wl.dtype, wl.n_tokens
     codec = Codec(dt, to_device(t["U"], dt), to_device(E0, dt), to_device(P0, dt))
@@ -202,8 +203,8 @@ def test_decompress_wire_large_batches(k, with_ids):
     wire = torch.from_numpy(wire_np).cuda()
     ids = torch.from_numpy(t["ids"]).cuda()
     Xh = codec.decompress_wire(wire, None if with_ids else ids, seq_len=wl.seq_len, with_ids=with_ids)
-    expect_kernel(B.SSN_KERNEL_UMMA_EXPAND,
-                  has=B.SSN_KVAR_E | B.SSN_KVAR_P | B.SSN_KVAR_ALT | (B.SSN_KVAR_WIDE if 2 * k > 64 else 0))
+    expect_kernel(B.SSN_KERNEL_UMMA_EXPAND, has=B.SSN_KVAR_E | B.SSN_KVAR_P | B.SSN_KVAR_ALT | B.SSN_KVAR_TWO_RUNS,
+                  lacks=B.SSN_KVAR_WIDE)
     Xo, _ = oracle.decompress(coords, f64(t["U"], dt), f64(E0, dt), t["ids"], f64(P0, dt),
                               oracle.token_positions(n, wl.seq_len))
     assert_close(host64(Xh, dt), Xo, dt, f"decompress_wire k={k}")
