@@ -245,7 +245,11 @@ struct UmmaProjectConfig {
   static_assert(kStagesN >= 2, "no room for two stages");
   static constexpr int kGatherLag = kStagesN > 3 ? 3 : kStagesN - 1;   // stages between issuing a gather and publishing it
   static constexpr int kAccCols = kN <= 32 ? 32 : (kN <= 64 ? 64 : 128);   // TMEM columns per accumulator
-  static constexpr int kIssuers = kATiles;                          // one MMA-issuing thread per A operand
+  // One MMA-issuing thread per A operand.  With X as the only operand two threads take alternate
+  // stages into an accumulator each (summed in the epilogue): one thread sustains a stage of four
+  // MMAs, a wait and a commit per ~540 clocks, two consume the ring at the rate of the tensor pipe.
+  static constexpr bool kSplitIssue = !HAS_E && !HAS_P;
+  static constexpr int kIssuers = kSplitIssue ? 2 : kATiles;
   static constexpr int kBufs = 2 * kIssuers * kAccCols <= 512 ? 2 : 1;   // accumulator sets (tiles in flight)
   // accumulator slots; with E and P and N <= 64 one more holds the shared positional product
   static constexpr int kAccSlots = kBufs * kIssuers + ((HAS_E && HAS_P && kN <= 64) ? 1 : 0);
@@ -388,7 +392,7 @@ codec_umma_project_kernel(const MmaArgs a, const __grid_constant__ UmmaMaps maps
     mbar_init(ring_free_bar, 4);
     for (int s = 0; s < S; ++s) {
       mbar_init(full_bar(s), HAS_E ? 5 : 1);
-      mbar_init(empty_bar(s), Cfg::kIssuers);
+      mbar_init(empty_bar(s), Cfg::kSplitIssue ? 1 : Cfg::kIssuers);   // a stage is read by all issuers, or by its own
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(acc_full_bar(b), Cfg::kIssuers);
@@ -455,7 +459,7 @@ codec_umma_project_kernel(const MmaArgs a, const __grid_constant__ UmmaMaps maps
     // accumulator, so that the three instruction streams issue side by side; the epilogue
     // combines X.U - E.U - P.U.  A stage is released when all issuers have committed.
     // warp 1 -> X; warp 10 -> the first table operand present; warp 11 -> P when both are present
-    const int which = warp == 1 ? 0 : (warp == 10 ? (Cfg::kATiles >= 2 ? 1 : -1) : (warp == 11 && Cfg::kATiles == 3 ? 2 : -1));
+    const int which = warp == 1 ? 0 : (warp == 10 ? (Cfg::kIssuers >= 2 ? 1 : -1) : (warp == 11 && Cfg::kIssuers == 3 ? 2 : -1));
     if (lane == 0 && which >= 0) {
       constexpr uint32_t idesc = umma_idesc(Cfg::kN, false);
       // A tiles: K-major rows of 128 bytes, 8-row groups 1024 bytes apart.  U slice: MN-major,
@@ -486,25 +490,30 @@ codec_umma_project_kernel(const MmaArgs a, const __grid_constant__ UmmaMaps maps
         const uint32_t d_tmem =
             tmem_base + (uint32_t)(p_issuer && pshare ? kPersistentAcc : buf * Cfg::kIssuers + which) * Cfg::kAccCols;
         for (int st = st_lo; st < st_hi; ++st) {
-          if (!dead && !mbar_wait(full_bar(slot), parity)) timed_out();
-          asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
-          const uint32_t base = smem0 + (uint32_t)slot * Cfg::kStageBytes;
-          // the start-address field (address / 16) is added to descriptors built once: a K step
-          // is 32 bytes of an A row and 16 rows = 2048 bytes of the U slice
-          const uint64_t adesc = adesc0 + umma_desc_addr(base + (uint32_t)which * Cfg::kATileBytes);
-          const uint64_t bdesc = bdesc0 + umma_desc_addr(base + Cfg::kATiles * Cfg::kATileBytes);
-          if (contract) {
+          // alternate stages when two threads share the one operand
+          const bool mine = !Cfg::kSplitIssue || ((st - st_lo) & 1) == which;
+          if (mine) {
+            if (!dead && !mbar_wait(full_bar(slot), parity)) timed_out();
+            asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+            const uint32_t base = smem0 + (uint32_t)slot * Cfg::kStageBytes;
+            // the start-address field (address / 16) is added to descriptors built once: a K step
+            // is 32 bytes of an A row and 16 rows = 2048 bytes of the U slice
+            const uint64_t adesc = adesc0 + umma_desc_addr(base + (uint32_t)(Cfg::kSplitIssue ? 0 : which) * Cfg::kATileBytes);
+            const uint64_t bdesc = bdesc0 + umma_desc_addr(base + Cfg::kATiles * Cfg::kATileBytes);
+            const int first_st = st_lo + (Cfg::kSplitIssue ? which : 0);   // this thread's first stage of the tile
+            if (contract) {
 #pragma unroll
-            for (int j = 0; j < kUmmaCols / 16; ++j)
-              umma_bf16(d_tmem, adesc + j * 2, bdesc + j * 128, idesc, (st > st_lo || j > 0) ? 1u : 0u);
+              for (int j = 0; j < kUmmaCols / 16; ++j)
+                umma_bf16(d_tmem, adesc + j * 2, bdesc + j * 128, idesc, (st > first_st || j > 0) ? 1u : 0u);
+            }
+            umma_commit(empty_bar(slot));
           }
-          umma_commit(empty_bar(slot));
-          if (st == st_hi - 1) umma_commit(acc_full_bar(buf));
           if (++slot == S) {
             slot = 0;
             parity ^= 1u;
           }
         }
+        umma_commit(acc_full_bar(buf));   // arrives when every MMA this thread issued for the tile is done
       }
     }
   } else if (warp < 6) {
@@ -581,7 +590,8 @@ codec_umma_project_kernel(const MmaArgs a, const __grid_constant__ UmmaMaps maps
       for (int q = 0; q < Cfg::kN / 16; ++q) tmem_ld16(taddr + q * 16, v[q]);
       asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
 #pragma unroll
-      for (int op = 1; op < Cfg::kIssuers; ++op) {   // Z = X.U - E.U - P.U
+      for (int op = 1; op < Cfg::kIssuers; ++op) {   // Z = X.U - E.U - P.U (or the two halves of X.U)
+        if (Cfg::kSplitIssue && st_hi - st_lo < 2) continue;   // a single stage: the second thread had none
         const bool is_p = HAS_P && op == kPTile;
         if (is_p && p_act == 2) continue;              // the peer subtracts the whole product
         // a sharing launch keeps P.U in its persistent accumulator
@@ -594,7 +604,9 @@ codec_umma_project_kernel(const MmaArgs a, const __grid_constant__ UmmaMaps maps
           tmem_ld16(oaddr + q * 16, w);
           asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
 #pragma unroll
-          for (int i = 0; i < 16; ++i) v[q][i] = __float_as_uint(__uint_as_float(v[q][i]) - __uint_as_float(w[i]));
+          for (int i = 0; i < 16; ++i)
+            v[q][i] = __float_as_uint(Cfg::kSplitIssue ? __uint_as_float(v[q][i]) + __uint_as_float(w[i])
+                                                       : __uint_as_float(v[q][i]) - __uint_as_float(w[i]));
         }
       }
       asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
