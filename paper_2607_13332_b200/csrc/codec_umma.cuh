@@ -8,11 +8,13 @@
 //
 //   warp 0   producer.  Per stage (128 tokens x 64 columns) one TMA box load of X, one of the
 //            P rows (positions of a tile are consecutive) and one of the 64 x k slice of U.
-//   warps 1, 10, 11  one thread each issues the tcgen05.mma (M=128, N=k rounded up to 16, K=16) of
-//            ONE A operand (X, E, P) into its own accumulator and commits to the stage's "empty"
-//            barrier (the tensor pipe retires one such instruction per ~87 clocks whatever
-//            its N).  The last stage of a tile also commits to the accumulators'
-//            "full" barrier.  Warp 1 owns the TMEM allocation.
+//   warps 1, 12, 10, 13, 11  one thread each issues tcgen05.mma (M=128, N=k rounded up to 16, K=16)
+//            into its own accumulator and commits to the stage's "empty" barrier (the tensor pipe
+//            retires one such instruction per ~87 clocks whatever its N): warps 1 and 12 the X
+//            operand on alternate stages, warps 10 and 13 the E operand likewise, warp 11 the P
+//            operand.  After a
+//            tile's last stage each commits to the accumulators' "full" barrier.  Warp 1 owns the
+//            TMEM allocation.
 //   warps 2-5  gather the E rows of the tile: 8 lanes copy one 128-byte row piece with cp.async
 //            straight into the swizzled tile, three stages ahead of the barrier arrival that
 //            publishes them (an id outside the table points at a row of zeros).
@@ -30,7 +32,7 @@
 
 namespace ssn {
 
-constexpr int kUmmaThreads = 384;
+constexpr int kUmmaThreads = 448;   // 14 warps, see the roles below
 constexpr int kUmmaTile = 128;     // tokens per tile (MMA M)
 constexpr int kUmmaCols = 64;      // columns of X per stage (one 128-byte swizzle row)
 constexpr int kWaitSpins = 1 << 22;
@@ -243,16 +245,27 @@ struct UmmaProjectConfig {
   static constexpr int kFit = (kMaxSmem - 1024 - 512) / kStageBytes;
   static constexpr int kStagesN = kFit < 10 ? kFit : 10;
   static_assert(kStagesN >= 2, "no room for two stages");
-  static constexpr int kGatherLag = kStagesN > 3 ? 3 : kStagesN - 1;   // stages between issuing a gather and publishing it
+  // Stages between issuing a gather and publishing it.  Two less than the ring: with a lag of S - 1
+  // the first stage is published only when every slot of the ring holds a pending gather, and the
+  // issuers starve (E and P, S = 4: 151 us with a lag of 3, 133 us with 2, 145 us with 1).
+  static constexpr int kGatherLag = kStagesN > 3 ? kStagesN - 2 : 1;
   static constexpr int kAccCols = kN <= 32 ? 32 : (kN <= 64 ? 64 : 128);   // TMEM columns per accumulator
-  // One MMA-issuing thread per A operand.  With X as the only operand two threads take alternate
-  // stages into an accumulator each (summed in the epilogue): one thread sustains a stage of four
-  // MMAs, a wait and a commit per ~540 clocks, two consume the ring at the rate of the tensor pipe.
-  static constexpr bool kSplitIssue = !HAS_E && !HAS_P;
-  static constexpr int kIssuers = kSplitIssue ? 2 : kATiles;
+  // MMA-issuing threads, each with an accumulator of its own.  One thread sustains a stage of
+  // four MMAs, a wait and a commit per ~540 clocks, which is slower than the ring can deliver and
+  // than the tensor pipe can run; so the X operand gets TWO threads that take alternate stages
+  // (their accumulators are summed in the epilogue) wherever tensor memory has room for it, and
+  // the E and P operands one thread each.
+  // E gets the same split as X whenever it is present: the two halves are then combined as
+  // (X0 - E0) + (X1 - E1), so that rows equal to their E rows still cancel exactly.
+  // (With E and P the five accumulators would leave one buffer of tensor memory; measured, the split
+  // gains nothing there: 135 against 133 us.)
+  static constexpr int kXIssuers = (!HAS_E || (kN <= 64 && !HAS_P)) ? 2 : 1;
+  static constexpr int kEIssuers = HAS_E ? kXIssuers : 0;
+  static constexpr int kIssuers = kXIssuers + kEIssuers + (HAS_P ? 1 : 0);
   static constexpr int kBufs = 2 * kIssuers * kAccCols <= 512 ? 2 : 1;   // accumulator sets (tiles in flight)
-  // accumulator slots; with E and P and N <= 64 one more holds the shared positional product
-  static constexpr int kAccSlots = kBufs * kIssuers + ((HAS_E && HAS_P && kN <= 64) ? 1 : 0);
+  // accumulator slots: kIssuers per buffer; a launch that shares the positional product keeps it
+  // in buffer 0's slot of the P issuer (buffer 1's stays unused then)
+  static constexpr int kAccSlots = kBufs * kIssuers;
   static constexpr int kTmemCols = (kAccSlots * kAccCols) <= 128 ? 128 : ((kAccSlots * kAccCols) <= 256 ? 256 : 512);
   static_assert(kAccSlots * kAccCols <= 512, "accumulators do not fit in tensor memory");
   static constexpr int kBarBytes = (2 * kStagesN + 6) * 8 + 16;
@@ -385,14 +398,14 @@ codec_umma_project_kernel(const MmaArgs a, const __grid_constant__ UmmaMaps maps
     cached_blk = -1;
     return rank0_has ? (cta_rank == 0 ? 1 : 2) : 0;
   };
-  constexpr int kPersistentAcc = 2 * Cfg::kIssuers;   // TMEM slot (of kAccCols columns) of the cached P U
+  constexpr int kPersistentAcc = Cfg::kIssuers - 1;   // TMEM slot of the cached P U: buffer 0's slot of the P issuer
 
   if (threadIdx.x == 0) {
     mbar_init(partial_ready_bar, 128);
     mbar_init(ring_free_bar, 4);
     for (int s = 0; s < S; ++s) {
       mbar_init(full_bar(s), HAS_E ? 5 : 1);
-      mbar_init(empty_bar(s), Cfg::kSplitIssue ? 1 : Cfg::kIssuers);   // a stage is read by all issuers, or by its own
+      mbar_init(empty_bar(s), Cfg::kATiles);   // one commit per operand (the X threads take turns)
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(acc_full_bar(b), Cfg::kIssuers);
@@ -455,11 +468,20 @@ codec_umma_project_kernel(const MmaArgs a, const __grid_constant__ UmmaMaps maps
     }
   } else if (warp == 1 || warp >= 10) {
     // ------------------------------------------------------------------------- MMA issuers
-    // One thread per A operand (X: warp 1, E: warp 10, P: warp 11), each with its own
-    // accumulator, so that the three instruction streams issue side by side; the epilogue
-    // combines X.U - E.U - P.U.  A stage is released when all issuers have committed.
-    // warp 1 -> X; warp 10 -> the first table operand present; warp 11 -> P when both are present
-    const int which = warp == 1 ? 0 : (warp == 10 ? (Cfg::kIssuers >= 2 ? 1 : -1) : (warp == 11 && Cfg::kIssuers == 3 ? 2 : -1));
+    // Issuer index `which` (= its accumulator slot in a buffer) and the A tile `opnd` it reads:
+    // warp 1 -> X; warp 12 -> X too (alternate stages) when kXIssuers == 2; warp 10 -> the first
+    // table operand present; warp 11 -> P when both are present.  The epilogue combines
+    // X.U - E.U - P.U.  A stage is released when every operand's issuer has committed.
+    // (warp 13 -> E on alternate stages when kEIssuers == 2)
+    const int which = warp == 1 ? 0
+                      : warp == 12 ? (Cfg::kXIssuers == 2 ? 1 : -1)
+                      : warp == 10 ? (HAS_E ? Cfg::kXIssuers : (HAS_P ? Cfg::kXIssuers : -1))
+                      : warp == 13 ? (Cfg::kEIssuers == 2 ? Cfg::kXIssuers + 1 : -1)
+                                   : (warp == 11 && HAS_E && HAS_P ? Cfg::kIssuers - 1 : -1);
+    const bool is_x = which < Cfg::kXIssuers, is_e = !is_x && which < Cfg::kXIssuers + Cfg::kEIssuers;
+    const int opnd = is_x ? 0 : (is_e ? 1 : kPTile);
+    const int half = is_x ? which : which - Cfg::kXIssuers;        // which of an operand's alternating threads
+    const int halves = is_x ? Cfg::kXIssuers : (is_e ? Cfg::kEIssuers : 1);
     if (lane == 0 && which >= 0) {
       constexpr uint32_t idesc = umma_idesc(Cfg::kN, false);
       // A tiles: K-major rows of 128 bytes, 8-row groups 1024 bytes apart.  U slice: MN-major,
@@ -469,7 +491,7 @@ codec_umma_project_kernel(const MmaArgs a, const __grid_constant__ UmmaMaps maps
       uint32_t parity = 0;
       int64_t tcount = 0;
       int64_t cached_blk = -1;
-      const bool p_issuer = HAS_P && which == kPTile;
+      const bool p_issuer = HAS_P && opnd == kPTile;
       for (int it = 0; it < my_tiles; ++it, ++tcount) {
         int64_t tile;
         int st_lo, st_hi;
@@ -491,16 +513,16 @@ codec_umma_project_kernel(const MmaArgs a, const __grid_constant__ UmmaMaps maps
             tmem_base + (uint32_t)(p_issuer && pshare ? kPersistentAcc : buf * Cfg::kIssuers + which) * Cfg::kAccCols;
         for (int st = st_lo; st < st_hi; ++st) {
           // alternate stages when two threads share the one operand
-          const bool mine = !Cfg::kSplitIssue || ((st - st_lo) & 1) == which;
+          const bool mine = halves == 1 || ((st - st_lo) & 1) == half;
           if (mine) {
             if (!dead && !mbar_wait(full_bar(slot), parity)) timed_out();
             asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
             const uint32_t base = smem0 + (uint32_t)slot * Cfg::kStageBytes;
             // the start-address field (address / 16) is added to descriptors built once: a K step
             // is 32 bytes of an A row and 16 rows = 2048 bytes of the U slice
-            const uint64_t adesc = adesc0 + umma_desc_addr(base + (uint32_t)(Cfg::kSplitIssue ? 0 : which) * Cfg::kATileBytes);
+            const uint64_t adesc = adesc0 + umma_desc_addr(base + (uint32_t)opnd * Cfg::kATileBytes);
             const uint64_t bdesc = bdesc0 + umma_desc_addr(base + Cfg::kATiles * Cfg::kATileBytes);
-            const int first_st = st_lo + (Cfg::kSplitIssue ? which : 0);   // this thread's first stage of the tile
+            const int first_st = st_lo + (halves == 2 ? half : 0);   // this thread's first stage of the tile
             if (contract) {
 #pragma unroll
               for (int j = 0; j < kUmmaCols / 16; ++j)
@@ -589,26 +611,40 @@ codec_umma_project_kernel(const MmaArgs a, const __grid_constant__ UmmaMaps maps
 #pragma unroll
       for (int q = 0; q < Cfg::kN / 16; ++q) tmem_ld16(taddr + q * 16, v[q]);
       asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
-#pragma unroll
-      for (int op = 1; op < Cfg::kIssuers; ++op) {   // Z = X.U - E.U - P.U (or the two halves of X.U)
-        if (Cfg::kSplitIssue && st_hi - st_lo < 2) continue;   // a single stage: the second thread had none
-        const bool is_p = HAS_P && op == kPTile;
-        if (is_p && p_act == 2) continue;              // the peer subtracts the whole product
-        // a sharing launch keeps P.U in its persistent accumulator
-        const uint32_t oaddr = is_p && pshare
-                                   ? tmem_base + ((uint32_t)(quarter * 32) << 16) + kPersistentAcc * Cfg::kAccCols
-                                   : taddr + op * Cfg::kAccCols;
+      // Z = (X0 - E0) + (X1 - E1) - P.U: slot 0 is X0 (in v); E0 follows the X slots
+      const bool two_halves = Cfg::kXIssuers == 2 && st_hi - st_lo >= 2;   // a single stage: the second threads had none
+      auto combine = [&](uint32_t addr, int sign) {     // v += sign * accumulator at addr
 #pragma unroll
         for (int q = 0; q < Cfg::kN / 16; ++q) {
           uint32_t w[16];
-          tmem_ld16(oaddr + q * 16, w);
+          tmem_ld16(addr + q * 16, w);
           asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
 #pragma unroll
           for (int i = 0; i < 16; ++i)
-            v[q][i] = __float_as_uint(Cfg::kSplitIssue ? __uint_as_float(v[q][i]) + __uint_as_float(w[i])
-                                                       : __uint_as_float(v[q][i]) - __uint_as_float(w[i]));
+            v[q][i] = __float_as_uint(sign > 0 ? __uint_as_float(v[q][i]) + __uint_as_float(w[i])
+                                               : __uint_as_float(v[q][i]) - __uint_as_float(w[i]));
+        }
+      };
+      if (HAS_E) combine(taddr + Cfg::kXIssuers * Cfg::kAccCols, -1);                    // X0 - E0
+      if (two_halves) {
+        if (Cfg::kEIssuers == 2) {                                                        // + (X1 - E1)
+#pragma unroll
+          for (int q = 0; q < Cfg::kN / 16; ++q) {
+            uint32_t x1[16], e1[16];
+            tmem_ld16(taddr + Cfg::kAccCols + q * 16, x1);
+            tmem_ld16(taddr + (Cfg::kXIssuers + 1) * Cfg::kAccCols + q * 16, e1);
+            asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
+#pragma unroll
+            for (int i = 0; i < 16; ++i)
+              v[q][i] = __float_as_uint(__uint_as_float(v[q][i]) + (__uint_as_float(x1[i]) - __uint_as_float(e1[i])));
+          }
+        } else {
+          combine(taddr + Cfg::kAccCols, +1);                                             // + X1
         }
       }
+      if (HAS_P && p_act != 2)   // 2: the peer subtracts the whole product; a sharing launch keeps P.U persistent
+        combine(pshare ? tmem_base + ((uint32_t)(quarter * 32) << 16) + kPersistentAcc * Cfg::kAccCols
+                       : taddr + (Cfg::kIssuers - 1) * Cfg::kAccCols, -1);
       asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory");
       __syncwarp();
       if (lane == 0) mbar_arrive(acc_empty_bar(buf));
