@@ -514,8 +514,13 @@ codec_umma_project_kernel(const MmaArgs a, const __grid_constant__ UmmaMaps maps
         for (int st = st_lo; st < st_hi; ++st) {
           // alternate stages when two threads share the one operand
           const bool mine = halves == 1 || ((st - st_lo) & 1) == half;
+          // Every issuer waits on EVERY stage, its partner's too.  A parity wait tells apart only
+          // the current phase of a barrier and the one before it: a thread that skipped its
+          // partner's stages could reach a slot while the load of the slot's previous use (a
+          // partner's stage, loads complete out of order) was still in flight, take that earlier
+          // phase for its own, consume a half-written stage and arrive on "empty" once too often.
+          if (!dead && !mbar_wait(full_bar(slot), parity)) timed_out();
           if (mine) {
-            if (!dead && !mbar_wait(full_bar(slot), parity)) timed_out();
             asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
             const uint32_t base = smem0 + (uint32_t)slot * Cfg::kStageBytes;
             // the start-address field (address / 16) is added to descriptors built once: a K step
