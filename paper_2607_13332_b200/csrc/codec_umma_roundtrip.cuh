@@ -17,8 +17,9 @@
 //           read it (one row per thread), round to bf16 into a swizzled staging slab and hand
 //           32 rows x 64 columns at a time to a TMA store, which also clips the rows past n.
 //
-//   warp 0  pass-1 producer     warp 1  MMA issuer, owns the TMEM allocation
+//   warp 0  pass-1 producer     warp 1  MMA issuer (pass 1: even stages; pass 2), owns the TMEM allocation
 //   warps 2-5  epilogue (TMEM lanes 32*(warp%4) ..)     warp 6  pass-2 producer (U chunks)
+//   warp 7  second pass-1 MMA issuer (odd stages, into the second half-accumulator of C)
 //
 // LEFT variant (W stored [d x m], the subspace on the rows: W <- U (U^T W)): a tile is a block of
 // 128 COLUMNS of W over all d rows.  Pass 1 contracts over the rows, T^T = W_blk^T U, with the block
@@ -79,8 +80,11 @@ struct UmmaRoundTripConfig {
   static constexpr int kFit = (kMaxSmem - 1024 - 512 - kFixedBytes) / kStageBytes;
   static constexpr int kStagesN = kFit < 8 ? kFit : 8;
   static_assert(kStagesN >= 2, "no room for two stages");
-  static constexpr int kAcc1Col = 0;                            // TMEM columns: C, then two D buffers
-  static constexpr int kDCol = 128;
+  // TMEM columns: C in two halves (pass 1 has two issuing threads on alternate stages, as in the
+  // projection kernel: one thread cannot issue as fast as the ring delivers), then two D buffers
+  static constexpr int kAcc1Col = 0;
+  static constexpr int kAcc1bCol = kN <= 64 ? 64 : 128;
+  static constexpr int kDCol = kN <= 64 ? 128 : 256;
   static constexpr int kTmemCols = 512;
   static constexpr int kBars = 2 * kStagesN + 2 + 2 * kU2Stages + 4;
   static constexpr int kSmemBytes = 1024 + kStagesN * kStageBytes + kFixedBytes + kBars * 8 + 16;
@@ -141,7 +145,7 @@ codec_umma_roundtrip_kernel(const MmaArgs a, const __grid_constant__ UmmaRoundTr
       mbar_init(full_bar(s), 1);
       mbar_init(empty_bar(s), 1);
     }
-    mbar_init(acc1_full_bar, 1);
+    mbar_init(acc1_full_bar, 2);   // both pass-1 issuers
     mbar_init(c_ready_bar, 4);
     for (int s = 0; s < S2; ++s) {
       mbar_init(u2_full_bar(s), 1);
@@ -239,14 +243,18 @@ codec_umma_roundtrip_kernel(const MmaArgs a, const __grid_constant__ UmmaRoundTr
       for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x, ++tcount) {
         const uint32_t acc1 = tmem_base + Cfg::kAcc1Col;
         for (int st = 0; st < nstage; ++st) {
+          // both pass-1 issuers wait on every stage (a thread that skipped a barrier's phase could
+          // take the phase before it for the one it wants); the odd stages are warp 7's
           if (!dead && !mbar_wait(full_bar(slot), parity)) timed_out();
-          asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
-          const uint32_t base = ring + (uint32_t)slot * Cfg::kStageBytes;
-          const uint64_t ad = (LEFT ? wdesc : kdesc) + umma_desc_addr(base), bd = udesc + umma_desc_addr(base + Cfg::kTileBytes);
+          if ((st & 1) == 0) {
+            asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+            const uint32_t base = ring + (uint32_t)slot * Cfg::kStageBytes;
+            const uint64_t ad = (LEFT ? wdesc : kdesc) + umma_desc_addr(base), bd = udesc + umma_desc_addr(base + Cfg::kTileBytes);
 #pragma unroll
-          for (int j = 0; j < kUmmaCols / 16; ++j)   // a K step: 32 bytes of a K-major row, 16 rows of an MN-major tile
-            umma_bf16(acc1, ad + j * (LEFT ? 128 : 2), bd + j * 128, idesc1, (st > 0 || j > 0) ? 1u : 0u);
-          umma_commit(empty_bar(slot));
+            for (int j = 0; j < kUmmaCols / 16; ++j)   // a K step: 32 bytes of a K-major row, 16 rows of an MN-major tile
+              umma_bf16(acc1, ad + j * (LEFT ? 128 : 2), bd + j * 128, idesc1, (st > 0 || j > 0) ? 1u : 0u);
+            umma_commit(empty_bar(slot));
+          }
           if (++slot == S) {
             slot = 0;
             parity ^= 1u;
@@ -284,6 +292,40 @@ codec_umma_roundtrip_kernel(const MmaArgs a, const __grid_constant__ UmmaRoundTr
         }
       }
     }
+  } else if (warp == 7) {
+    // ------------------------------------------------------------------------- second pass-1 issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc1 = umma_idesc(Cfg::kN, false) | (LEFT ? (1u << 15) : 0u);
+      const uint64_t kdesc = umma_desc(0, 16, 1024, 2);
+      const uint64_t udesc = umma_desc(0, Cfg::kUGroupBytes, 1024, 2);
+      const uint64_t wdesc = umma_desc(0, Cfg::kTileBytes / 2, 1024, 2);
+      int slot = 0;
+      uint32_t parity = 0;
+      int64_t tcount = 0;
+      for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x, ++tcount) {
+        const uint32_t acc1b = tmem_base + Cfg::kAcc1bCol;
+        for (int st = 0; st < nstage; ++st) {
+          if (!dead && !mbar_wait(full_bar(slot), parity)) timed_out();
+          if ((st & 1) == 1) {
+            asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+            const uint32_t base = ring + (uint32_t)slot * Cfg::kStageBytes;
+            const uint64_t ad = (LEFT ? wdesc : kdesc) + umma_desc_addr(base), bd = udesc + umma_desc_addr(base + Cfg::kTileBytes);
+#pragma unroll
+            for (int j = 0; j < kUmmaCols / 16; ++j)
+              umma_bf16(acc1b, ad + j * (LEFT ? 128 : 2), bd + j * 128, idesc1, (st > 1 || j > 0) ? 1u : 0u);
+            umma_commit(empty_bar(slot));
+          }
+          if (++slot == S) {
+            slot = 0;
+            parity ^= 1u;
+          }
+        }
+        umma_commit(acc1_full_bar);
+        // the epilogue must have read this tile's half before the next tile's MMAs overwrite it
+        if (!dead && !mbar_wait(c_ready_bar, (uint32_t)(tcount & 1))) timed_out();
+        asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
+      }
+    }
   } else if (warp >= 2 && warp < 6) {
     // ------------------------------------------------------------------------- epilogue
     const int quarter = warp & 3;   // the TMEM lanes this warp may read: 32*quarter .. +31
@@ -305,6 +347,16 @@ codec_umma_roundtrip_kernel(const MmaArgs a, const __grid_constant__ UmmaRoundTr
 #pragma unroll
         for (int q = 0; q < Cfg::kN / 16; ++q) tmem_ld16(lane_addr + Cfg::kAcc1Col + q * 16, v[q]);
         asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
+        if (nstage >= 2) {   // the odd stages' half (with a single stage it was never written)
+#pragma unroll
+          for (int q = 0; q < Cfg::kN / 16; ++q) {
+            uint32_t w[16];
+            tmem_ld16(lane_addr + Cfg::kAcc1bCol + q * 16, w);
+            asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
+#pragma unroll
+            for (int i = 0; i < 16; ++i) v[q][i] = __float_as_uint(__uint_as_float(v[q][i]) + __uint_as_float(w[i]));
+          }
+        }
         const int64_t t = row0 + r;
 #pragma unroll
         for (int c = 0; c < 8 * Cfg::kKG; ++c) {           // 16-byte pieces: 8 coordinates each
