@@ -8,18 +8,19 @@
 //
 //   warp 0   producer.  Per stage (128 tokens x 64 columns) one TMA box load of X, one of the
 //            P rows (positions of a tile are consecutive) and one of the 64 x k slice of U.
-//   warps 1, 12, 10, 13, 11  one thread each issues tcgen05.mma (M=128, N=k rounded up to 16, K=16)
-//            into its own accumulator and commits to the stage's "empty" barrier (the tensor pipe
-//            retires one such instruction per ~87 clocks whatever its N): warps 1 and 12 the X
-//            operand on alternate stages, warps 10 and 13 the E operand likewise, warp 11 the P
-//            operand.  After a
-//            tile's last stage each commits to the accumulators' "full" barrier.  Warp 1 owns the
-//            TMEM allocation.
-//   warps 2-5  gather the E rows of the tile: 8 lanes copy one 128-byte row piece with cp.async
-//            straight into the swizzled tile, three stages ahead of the barrier arrival that
-//            publishes them (an id outside the table points at a row of zeros).
-//   warps 6-9  epilogue: tcgen05.ld their 32 TMEM lanes (one token per thread), round to bf16,
-//            store the Z rows; two accumulators let a tile's epilogue overlap the next tile's MMAs.
+//   warps 1-3 (and 12)  MMA issuers: one thread each issues tcgen05.mma (M=128, N=k rounded up to
+//            16, K=16) into its own accumulator and commits to the stage's "empty" barrier (the
+//            tensor pipe retires one such instruction per ~87 clocks whatever its N).  In the
+//            order X, X, E, E, P: an operand with two threads has them take alternate stages.
+//            After a tile's last stage each commits to the accumulators' "full" barrier.  Warp 1
+//            owns the TMEM allocation.
+//   warps 4-7  epilogue: tcgen05.ld their 32 TMEM lanes (one token per thread), combine the
+//            accumulators, round to bf16, store the Z rows; two sets of accumulators let a tile's
+//            epilogue overlap the next tile's MMAs.
+//   warps 8-11 (with E rows only)  gather the E rows of the tile: 8 lanes copy one 128-byte row
+//            piece with cp.async straight into the swizzled tile, some stages ahead of the
+//            barrier arrival that publishes them (an id outside the table points at a row of zeros).
+//   A launch carries only the warps its roles need (8, 12 or 13).
 //
 // X, E and P tiles use the 128-byte swizzled K-major layout (rows of 128 bytes); U arrives as a
 // 128-byte swizzled MN-major operand straight from its row-major storage.  Every wait is
@@ -32,7 +33,6 @@
 
 namespace ssn {
 
-constexpr int kUmmaThreads = 448;   // 14 warps, see the roles below
 constexpr int kUmmaTile = 128;     // tokens per tile (MMA M)
 constexpr int kUmmaCols = 64;      // columns of X per stage (one 128-byte swizzle row)
 constexpr int kWaitSpins = 1 << 22;
@@ -262,6 +262,12 @@ struct UmmaProjectConfig {
   static constexpr int kXIssuers = (!HAS_E || (kN <= 64 && !HAS_P)) ? 2 : 1;
   static constexpr int kEIssuers = HAS_E ? kXIssuers : 0;
   static constexpr int kIssuers = kXIssuers + kEIssuers + (HAS_P ? 1 : 0);
+  // Warps: 0 producer; 1-3 the first three issuers; 4-7 epilogue; with E rows 8-11 gather them and
+  // warp 12 is the fourth issuer (E only, k <= 64).  A launch has only the warps its roles need, so
+  // that the register budget of the epilogue (a whole accumulator row per thread) is not cut by
+  // warps that would idle: 256 threads without E rows, 384 or 416 with them.
+  static constexpr int kWarps = !HAS_E ? 8 : (kIssuers == 4 ? 13 : 12);
+  static constexpr int kThreads = 32 * kWarps;
   static constexpr int kBufs = 2 * kIssuers * kAccCols <= 512 ? 2 : 1;   // accumulator sets (tiles in flight)
   // accumulator slots: kIssuers per buffer; a launch that shares the positional product keeps it
   // in buffer 0's slot of the P issuer (buffer 1's stays unused then)
@@ -318,7 +324,7 @@ cudaError_t launch_tile_pairs(Kernel kernel, int threads, int smem, const MmaArg
 }
 
 template <int NTP, bool HAS_E, bool HAS_P>
-__global__ void __launch_bounds__(kUmmaThreads, 1)
+__global__ void __launch_bounds__((UmmaProjectConfig<NTP, HAS_E, HAS_P>::kThreads), 1)
 codec_umma_project_kernel(const MmaArgs a, const __grid_constant__ UmmaMaps maps) {
   using Cfg = UmmaProjectConfig<NTP, HAS_E, HAS_P>;
   constexpr int kETile = 1, kPTile = HAS_E ? 2 : 1;   // order of the tiles inside a stage
@@ -466,23 +472,18 @@ codec_umma_project_kernel(const MmaArgs a, const __grid_constant__ UmmaMaps maps
         }
       }
     }
-  } else if (warp == 1 || warp >= 10) {
+  } else if (warp < 4 || warp == 12) {
     // ------------------------------------------------------------------------- MMA issuers
-    // Issuer index `which` (= its accumulator slot in a buffer) and the A tile `opnd` it reads:
-    // warp 1 -> X; warp 12 -> X too (alternate stages) when kXIssuers == 2; warp 10 -> the first
-    // table operand present; warp 11 -> P when both are present.  The epilogue combines
-    // X.U - E.U - P.U.  A stage is released when every operand's issuer has committed.
-    // (warp 13 -> E on alternate stages when kEIssuers == 2)
-    const int which = warp == 1 ? 0
-                      : warp == 12 ? (Cfg::kXIssuers == 2 ? 1 : -1)
-                      : warp == 10 ? (HAS_E ? Cfg::kXIssuers : (HAS_P ? Cfg::kXIssuers : -1))
-                      : warp == 13 ? (Cfg::kEIssuers == 2 ? Cfg::kXIssuers + 1 : -1)
-                                   : (warp == 11 && HAS_E && HAS_P ? Cfg::kIssuers - 1 : -1);
+    // Issuer index `which` (= its accumulator slot in a buffer) and the A tile `opnd` it reads, in
+    // the order X, X again (alternate stages) when kXIssuers == 2, E, E again when kEIssuers == 2,
+    // P.  The epilogue combines X.U - E.U - P.U.  A stage is released when every operand's issuer
+    // has committed.
+    const int which = warp == 12 ? 3 : warp - 1;   // issuer index = its accumulator slot in a buffer
     const bool is_x = which < Cfg::kXIssuers, is_e = !is_x && which < Cfg::kXIssuers + Cfg::kEIssuers;
     const int opnd = is_x ? 0 : (is_e ? 1 : kPTile);
     const int half = is_x ? which : which - Cfg::kXIssuers;        // which of an operand's alternating threads
     const int halves = is_x ? Cfg::kXIssuers : (is_e ? Cfg::kEIssuers : 1);
-    if (lane == 0 && which >= 0) {
+    if (lane == 0 && which < Cfg::kIssuers) {
       constexpr uint32_t idesc = umma_idesc(Cfg::kN, false);
       // A tiles: K-major rows of 128 bytes, 8-row groups 1024 bytes apart.  U slice: MN-major,
       // 64-column groups kUGroupBytes apart, 8-row groups 1024 bytes apart.
@@ -543,10 +544,10 @@ codec_umma_project_kernel(const MmaArgs a, const __grid_constant__ UmmaMaps maps
         umma_commit(acc_full_bar(buf));   // arrives when every MMA this thread issued for the tile is done
       }
     }
-  } else if (warp < 6) {
+  } else if (warp >= 8) {
     // ------------------------------------------------------------------------- E row gather
     if (HAS_E) {
-      const int gw = warp - 2;                 // rows 32*gw .. 32*gw+31 of the tile
+      const int gw = warp - 8;                 // rows 32*gw .. 32*gw+31 of the tile
       const int piece = lane & 7, sub = lane >> 3;
       int slot = 0, pub_slot = 0, pending = 0;
       uint32_t parity = 1;

@@ -17,7 +17,7 @@ cudaError_t launch_umma_one(const MmaArgs &a, const UmmaMaps &maps, int sm_count
   }
   note_kernel(SSN_KERNEL_UMMA_PROJECT, (HAS_E ? SSN_KVAR_E : 0) | (HAS_P ? SSN_KVAR_P : 0) |
                                            (NTP > 8 ? SSN_KVAR_WIDE : 0) | (a.pshare ? SSN_KVAR_ALT : 0));
-  return launch_tile_pairs(kernel, kUmmaThreads, smem, a, maps, sm_count, stream);
+  return launch_tile_pairs(kernel, UmmaProjectConfig<NTP, HAS_E, HAS_P>::kThreads, smem, a, maps, sm_count, stream);
 }
 
 template <int NTP>
