@@ -19,24 +19,36 @@ from tests.harness import Codec
 pytestmark = pytest.mark.gpu
 
 DT = synth.BF16
-D, K, SEQ, NSEQ = 4096, 40, 2048, 32
+D, SEQ, NSEQ = 4096, 2048, 32
 STEPS, ROUNDS = 300, 4
 
+# (rank, E rows, P rows, prepared tables): the benchmark's two step variants, then the projection
+# kernel's other issuer layouts (E alone: four issuing threads on a ring of five; P alone; k = 128:
+# accumulators of 128 columns, one set only when E and P are operands)
+CASES = {
+    "rows": (40, True, True, False),
+    "prepared_tables": (40, True, True, True),
+    "embedding_only": (40, True, False, False),
+    "positions_only": (40, False, True, False),
+    "rank_128": (128, True, True, False),
+}
 
-@pytest.mark.parametrize("tables", [False, True], ids=["rows", "prepared_tables"])
-def test_queued_steps_after_idle_gaps_repeat_the_first_step(tables):
+
+@pytest.mark.parametrize("case", list(CASES))
+def test_queued_steps_after_idle_gaps_repeat_the_first_step(case):
+    k, with_e, with_p, tables = CASES[case]
     n = SEQ * NSEQ
     gen = synth_device.generator(77)
-    E = synth_device.embedding_table(synth_device.SWEEP_VOCAB, D, gen)
-    P = synth_device.positions_table(SEQ, D)
-    U = synth_device.basis(D, K, 1)
+    E = synth_device.embedding_table(synth_device.SWEEP_VOCAB, D, gen) if with_e else None
+    P = synth_device.positions_table(SEQ, D) if with_p else None
+    U = synth_device.basis(D, k, 1)
     X = synth_device.activations(n, D, gen)
     G = synth_device.activations(n, D, gen)
     ids = torch.from_numpy(synth.zipf_ids(n, synth_device.SWEEP_VOCAB, 1.1, seed=5)).cuda()
     codec = Codec(DT, U, E, P)
     if tables:
         codec.prepare_tables()
-    Z = torch.empty((n, K), dtype=torch.bfloat16, device="cuda")
+    Z = torch.empty((n, k), dtype=torch.bfloat16, device="cuda")
     dZ = torch.empty_like(Z)
     Xh = torch.empty_like(X)
     # the weights are re-projected in place step after step (projecting twice gives the same weight
