@@ -86,12 +86,13 @@ struct UmmaExpandConfig {
   static constexpr int kFixedBytes =
       kZBufs * kZBytes + kSelBytes + kUStages * kUStageBytes + kStagingBytes;
   static constexpr int kMaxSmem = 227 * 1024;
-  static constexpr int kEFit = (kMaxSmem - 1024 - 512 - kFixedBytes) / kEStageBytes;
+  static constexpr int kEFit = (kMaxSmem - 1024 - 1024 - kFixedBytes) / kEStageBytes;
   static constexpr int kEStages = HAS_E ? (kEFit < 12 ? kEFit : 12) : 0;
   static_assert(!HAS_E || kEStages >= 4, "no room for the E ring");
+  static constexpr int kDBufs = 2;                 // accumulators of 128 columns: one per epilogue group
   static constexpr int kTmemCols = 256;
   static constexpr int SE = HAS_E ? kEStages : 1;
-  static constexpr int kBars = 4 + 2 * kUStages + 2 * SE + 4;
+  static constexpr int kBars = 4 + 2 * kUStages + 8 * SE + 2 * kDBufs;   // the E ring has a full and an empty barrier per stage and QUARTER
   static constexpr int kSmemBytes = 1024 + kFixedBytes + kEStages * kEStageBytes + kBars * 8 + 16;
   static_assert(kSmemBytes <= kMaxSmem, "the rings do not fit in shared memory");
 };
@@ -140,10 +141,12 @@ codec_umma_expand_kernel(const MmaArgs a, const ExpandGeometry geo, const __grid
   auto z_empty_bar = [&](int b) { return bars + (2 + b) * 8; };
   auto u_full_bar = [&](int s) { return bars + (4 + s) * 8; };
   auto u_empty_bar = [&](int s) { return bars + (4 + SU + s) * 8; };
-  auto e_full_bar = [&](int s) { return bars + (4 + 2 * SU + s) * 8; };
-  auto e_empty_bar = [&](int s) { return bars + (4 + 2 * SU + SE + s) * 8; };
-  auto d_full_bar = [&](int b) { return bars + (4 + 2 * SU + 2 * SE + b) * 8; };
-  auto d_empty_bar = [&](int b) { return bars + (4 + 2 * SU + 2 * SE + 2 + b) * 8; };
+  // The E ring is handed over per QUARTER of a stage (32 rows: one gather warp fills them, one
+  // epilogue warp of either group consumes them), so that a late row holds up only its own quarter.
+  auto e_full_bar = [&](int s, int q) { return bars + (4 + 2 * SU + 4 * s + q) * 8; };
+  auto e_empty_bar = [&](int s, int q) { return bars + (4 + 2 * SU + 4 * SE + 4 * s + q) * 8; };
+  auto d_full_bar = [&](int b) { return bars + (4 + 2 * SU + 8 * SE + b) * 8; };
+  auto d_empty_bar = [&](int b) { return bars + (4 + 2 * SU + 8 * SE + Cfg::kDBufs + b) * 8; };
   const uint32_t tmem_slot = bars + Cfg::kBars * 8;
   volatile uint32_t *tmem_slot_ptr =
       reinterpret_cast<volatile uint32_t *>(smem_raw + (tmem_slot - smem_u32(smem_raw)));
@@ -172,6 +175,8 @@ codec_umma_expand_kernel(const MmaArgs a, const ExpandGeometry geo, const __grid
     for (int b = 0; b < 2; ++b) {
       mbar_init(z_full_bar(b), 1);
       mbar_init(z_empty_bar(b), 1);
+    }
+    for (int b = 0; b < Cfg::kDBufs; ++b) {
       mbar_init(d_full_bar(b), 1);
       mbar_init(d_empty_bar(b), 4);
     }
@@ -180,8 +185,10 @@ codec_umma_expand_kernel(const MmaArgs a, const ExpandGeometry geo, const __grid
       mbar_init(u_empty_bar(s), 1);
     }
     for (int s = 0; s < SE; ++s) {
-      mbar_init(e_full_bar(s), kGatherWarps * 32);   // one arrival per gather thread
-      mbar_init(e_empty_bar(s), 4);
+      for (int q = 0; q < 4; ++q) {
+        mbar_init(e_full_bar(s, q), 32);             // one arrival per thread of the quarter's gather warp
+        mbar_init(e_empty_bar(s, q), 1);             // the epilogue warp that consumed the quarter
+      }
     }
     asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
   }
@@ -286,8 +293,8 @@ codec_umma_expand_kernel(const MmaArgs a, const ExpandGeometry geo, const __grid
         int q0, q1;
         chunk_range(tile, q0, q1);
         for (int q = q0; q < q1; ++q, ++ccount) {
-          const int db = (int)(ccount & 1);
-          if (!dead && !mbar_wait(d_empty_bar(db), (uint32_t)(((ccount >> 1) & 1) ^ 1))) timed_out();
+          const int db = (int)(ccount % Cfg::kDBufs);
+          if (!dead && !mbar_wait(d_empty_bar(db), (uint32_t)(((ccount / Cfg::kDBufs) & 1) ^ 1))) timed_out();
           if (!dead && !mbar_wait(u_full_bar(slot), parity)) timed_out();
           asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
           const uint32_t base = u_ring + (uint32_t)slot * Cfg::kUStageBytes;
@@ -346,11 +353,11 @@ codec_umma_expand_kernel(const MmaArgs a, const ExpandGeometry geo, const __grid
         int q0, q1;
         chunk_range(tile, q0, q1);
         for (int qg = 2 * q0; qg < 2 * q1; ++qg) {     // 64-column groups of the row
-          if (!dead && !mbar_wait(e_empty_bar(slot), parity)) timed_out();
+          if (!dead && !mbar_wait(e_empty_bar(slot, gw), parity)) timed_out();
           const uint32_t base = e_ring + (uint32_t)slot * Cfg::kEStageBytes;
 #pragma unroll
           for (int i = 0; i < 8; ++i) cp_async16_cg(base + dst[i], src[i] + qg * 128);
-          asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];\n" ::"r"(e_full_bar(slot)) : "memory");
+          asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];\n" ::"r"(e_full_bar(slot, gw)) : "memory");
           if (++slot == SE) {
             slot = 0;
             parity ^= 1u;
@@ -386,8 +393,8 @@ codec_umma_expand_kernel(const MmaArgs a, const ExpandGeometry geo, const __grid
       for (int q = q0; q < q1; ++q, ++ccount) {
         if ((int)(ccount & 1) != group) continue;
         float ss = 0.f;   // sum of squares of this row's 128 columns of the chunk, before rounding
-        const int db = group;
-        if (!dead && !mbar_wait(d_full_bar(db), (uint32_t)((ccount >> 1) & 1))) timed_out();
+        const int db = (int)(ccount % Cfg::kDBufs);   // the group's accumulators alternate
+        if (!dead && !mbar_wait(d_full_bar(db), (uint32_t)((ccount / Cfg::kDBufs) & 1))) timed_out();
         asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
 #pragma unroll
         for (int g = 0; g < kChunkCols / 64; ++g) {
@@ -404,7 +411,7 @@ codec_umma_expand_kernel(const MmaArgs a, const ExpandGeometry geo, const __grid
           }
           uint32_t slab;   // 32 rows x 128 B handed to the TMA store
           if (HAS_E) {
-            if (!dead && !mbar_wait(e_full_bar(eslot), (uint32_t)((ecount / SE) & 1))) timed_out();
+            if (!dead && !mbar_wait(e_full_bar(eslot, quarter), (uint32_t)((ecount / SE) & 1))) timed_out();
             slab = e_ring + (uint32_t)eslot * Cfg::kEStageBytes + (uint32_t)quarter * 4096;
           } else {
             // the store that last read this slab (two stores ago) must be done reading it
@@ -454,11 +461,11 @@ codec_umma_expand_kernel(const MmaArgs a, const ExpandGeometry geo, const __grid
               // two chunks away and the stage would sit idle until then
               if (g == kChunkCols / 64 - 1) {
                 bulk_wait_read<0>();
-                if (held >= 0) mbar_arrive(e_empty_bar(held));
-                mbar_arrive(e_empty_bar(eslot));
+                if (held >= 0) mbar_arrive(e_empty_bar(held, quarter));
+                mbar_arrive(e_empty_bar(eslot, quarter));
               } else {
                 bulk_wait_read<1>();
-                if (held >= 0) mbar_arrive(e_empty_bar(held));
+                if (held >= 0) mbar_arrive(e_empty_bar(held, quarter));
               }
             }
           }
@@ -469,7 +476,7 @@ codec_umma_expand_kernel(const MmaArgs a, const ExpandGeometry geo, const __grid
     }
     if (HAS_E && lane == 0) {
       bulk_wait_read<0>();
-      if (held >= 0) mbar_arrive(e_empty_bar(held));
+      if (held >= 0) mbar_arrive(e_empty_bar(held, quarter));
     }
     if (lane == 0) bulk_wait<0>();
   }
