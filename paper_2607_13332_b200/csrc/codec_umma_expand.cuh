@@ -27,6 +27,9 @@
 //              swizzled stages (an id outside the table points at a row of zeros); the epilogue
 //              forms the sum in place and the stage is the source of the TMA store; a stage
 //              goes back to the gather warps as soon as the chunk's last store has read it.
+//              The ring is handed over per quarter of a stage (32 rows): gather warp q fills the
+//              rows that epilogue warp q of either group reads, and each quarter has its own
+//              pair of barriers.
 // L2: the output is stored with an evict_first policy and the P rows are loaded with evict_last,
 // so that the streams do not push the 16 rows under a chunk out before the next group of
 // sequences needs them.
