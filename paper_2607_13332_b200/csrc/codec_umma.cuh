@@ -349,10 +349,11 @@ codec_umma_project_kernel(const MmaArgs a, const __grid_constant__ UmmaMaps maps
 
   // Tile schedule.  The CTAs run as pairs (clusters of two).  Pair c takes the tiles c, c + pairs,
   // c + 2 pairs, ...; its two CTAs take them alternately, and when their number is odd the last
-  // tile is SPLIT: rank 0 contracts the first half of d, rank 1 the second half, rank 1 sends its
-  // fp32 partial sums into rank 0's (by then idle) stage ring through distributed shared memory,
-  // and rank 0 adds them and stores.  512 tiles on 74 pairs are 3 or 3.5 tiles per CTA instead of
-  // 3 or 4.  A launch without clusters is the same schedule with pairs of one CTA and no split.
+  // tile is SPLIT: rank 0 contracts the first half of d, rank 1 the second half; then each sends
+  // the fp32 partial sums of the 64 rows the OTHER finishes into that CTA's (by then idle) stage
+  // ring through distributed shared memory, adds what it receives for its own 64 rows and stores
+  // them.  512 tiles on 74 pairs are 3 or 3.5 tiles per CTA instead of 3 or 4.  A launch without
+  // clusters is the same schedule with pairs of one CTA and no split.
   uint32_t cluster_size, cta_rank;
   asm volatile("mov.u32 %0, %%cluster_nctaid.x;\n" : "=r"(cluster_size));
   asm volatile("mov.u32 %0, %%cluster_ctarank;\n" : "=r"(cta_rank));
@@ -407,8 +408,8 @@ codec_umma_project_kernel(const MmaArgs a, const __grid_constant__ UmmaMaps maps
   constexpr int kPersistentAcc = Cfg::kIssuers - 1;   // TMEM slot of the cached P U: buffer 0's slot of the P issuer
 
   if (threadIdx.x == 0) {
-    mbar_init(partial_ready_bar, 128);
-    mbar_init(ring_free_bar, 4);
+    mbar_init(partial_ready_bar, 64);   // the threads of the peer's two sending warps
+    mbar_init(ring_free_bar, 2);        // the peer's two receiving warps
     for (int s = 0; s < S; ++s) {
       mbar_init(full_bar(s), HAS_E ? 5 : 1);
       mbar_init(empty_bar(s), Cfg::kATiles);   // one commit per operand (the X threads take turns)
@@ -656,13 +657,17 @@ codec_umma_project_kernel(const MmaArgs a, const __grid_constant__ UmmaMaps maps
       if (lane == 0) mbar_arrive(acc_empty_bar(buf));
 
       if (split) {
-        // the split tile is the last one of both CTAs: every stage of rank 0's ring has been
-        // consumed once its accumulator is complete, so the ring can carry the partial sums
+        // The split tile is the last one of both CTAs, and each finishes HALF of its rows: rank 0
+        // the rows 0..63 (epilogue warps of quarters 0 and 1), rank 1 the rows 64..127.  A warp
+        // either receives the peer's partial sums of its rows or sends its own to the peer.  Every
+        // stage of a CTA's ring has been consumed once its accumulators are complete, so the ring
+        // can carry the 64 rows it receives.
         const uint32_t row_off = (uint32_t)(quarter * 32 + lane) * (Cfg::kN * 4);
-        if (cta_rank == 0) {
-          if (lane == 0) {
+        const uint32_t peer = cta_rank ^ 1u;
+        if ((uint32_t)(quarter >> 1) == cta_rank) {
+          if (lane == 0) {   // this CTA's ring is idle: the peer may write into it
             uint32_t remote;
-            asm volatile("mapa.shared::cluster.u32 %0, %1, %2;\n" : "=r"(remote) : "r"(ring_free_bar), "r"(1));
+            asm volatile("mapa.shared::cluster.u32 %0, %1, %2;\n" : "=r"(remote) : "r"(ring_free_bar), "r"(peer));
             asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];\n" ::"r"(remote) : "memory");
           }
           if (!dead && !mbar_wait_cluster(partial_ready_bar, 0)) timed_out();
@@ -681,8 +686,8 @@ codec_umma_project_kernel(const MmaArgs a, const __grid_constant__ UmmaMaps maps
         } else {
           if (!dead && !mbar_wait_cluster(ring_free_bar, 0)) timed_out();
           uint32_t remote_ring, remote_bar;
-          asm volatile("mapa.shared::cluster.u32 %0, %1, %2;\n" : "=r"(remote_ring) : "r"(smem0 + row_off), "r"(0));
-          asm volatile("mapa.shared::cluster.u32 %0, %1, %2;\n" : "=r"(remote_bar) : "r"(partial_ready_bar), "r"(0));
+          asm volatile("mapa.shared::cluster.u32 %0, %1, %2;\n" : "=r"(remote_ring) : "r"(smem0 + row_off), "r"(peer));
+          asm volatile("mapa.shared::cluster.u32 %0, %1, %2;\n" : "=r"(remote_bar) : "r"(partial_ready_bar), "r"(peer));
 #pragma unroll
           for (int q = 0; q < Cfg::kN / 16; ++q)
 #pragma unroll
@@ -690,7 +695,7 @@ codec_umma_project_kernel(const MmaArgs a, const __grid_constant__ UmmaMaps maps
               asm volatile("st.shared::cluster.v4.b32 [%0], {%1,%2,%3,%4};\n" ::"r"(remote_ring + (q * 16 + i) * 4),
                            "r"(v[q][i]), "r"(v[q][i + 1]), "r"(v[q][i + 2]), "r"(v[q][i + 3]) : "memory");
           asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];\n" ::"r"(remote_bar) : "memory");
-          continue;   // rank 0 stores this tile
+          continue;   // the peer stores these rows
         }
       }
 
