@@ -172,9 +172,12 @@ def test_project_and_roundtrip_mma_sync_large_batches(k):
 
 
 # ---- the projection kernel at large batches: shared positional product, ragged tail ---------------
+# (widths of 1 and 3 stages: a tile whose second issuing threads get no stage of their own, and an
+# odd number of stages for the two threads of an operand and for the two CTAs of a pair to share)
+@pytest.mark.parametrize("d", [64, 192, 256])
 @pytest.mark.parametrize("tables", ["EP", "E", "P", "none"])
-def test_compress_tcgen05_large_batches(tables):
-    wl, t, E0, P0 = _inputs(160, 128, 256, 40, 900, seed=3, tables=tables)
+def test_compress_tcgen05_large_batches(tables, d):
+    wl, t, E0, P0 = _inputs(160, 128, d, 40, 900, seed=3, tables=tables)
     dt, n = wl.dtype, wl.n_tokens
     codec = Codec(dt, to_device(t["U"], dt), to_device(E0, dt), to_device(P0, dt))
     ids = torch.from_numpy(t["ids"]).cuda()
