@@ -89,6 +89,41 @@ cudaError_t allow_dynamic_smem(Kernel kernel, int smem, std::atomic<uint64_t> &d
   return e;
 }
 
+// Launch of a tcgen05 kernel that may START before the kernel in front of it in the stream has
+// ended (programmatic dependent launch): its CTAs set up their barriers and tensor memory on the SMs
+// the earlier kernel has left, and wait (griddepcontrol.wait, which every such kernel executes after
+// its set-up and before it touches global memory) until that kernel is complete and its writes are
+// visible.  The earlier kernel allows this at its start (griddepcontrol.launch_dependents); behind
+// any other kernel, and inside a stream capture, the launch is an ordinary one.  cluster = 2 launches
+// pairs of CTAs.
+template <typename Kernel, typename... Args>
+cudaError_t launch_dependent(Kernel kernel, unsigned grid, int threads, int smem, cudaStream_t stream, int cluster,
+                             Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3((unsigned)threads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[2];
+  int n = 0;
+  if (cluster > 1) {
+    attr[n].id = cudaLaunchAttributeClusterDimension;
+    attr[n].val.clusterDim.x = (unsigned)cluster;
+    attr[n].val.clusterDim.y = 1;
+    attr[n].val.clusterDim.z = 1;
+    ++n;
+  }
+  cudaStreamCaptureStatus capturing = cudaStreamCaptureStatusNone;
+  if (cudaStreamIsCapturing(stream, &capturing) == cudaSuccess && capturing == cudaStreamCaptureStatusNone) {
+    attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[n].val.programmaticStreamSerializationAllowed = 1;
+    ++n;
+  }
+  cfg.attrs = attr;
+  cfg.numAttrs = n;
+  return cudaLaunchKernelEx(&cfg, kernel, args...);
+}
+
 // The tcgen05 kernels one by one; each returns cudaErrorNotSupported, with nothing launched, for
 // shapes and alignments that are not its own (the conditions are stated at the definitions).
 cudaError_t launch_codec_umma_project(const MmaArgs &a, bool shift, int sm_count, cudaStream_t stream);

@@ -298,29 +298,14 @@ cudaError_t launch_tile_pairs(Kernel kernel, int threads, int smem, const MmaArg
   const int64_t ntiles = (a.n + kUmmaTile - 1) / kUmmaTile;
   int64_t pairs = ntiles;   // with few tiles every pair has one and splits it over d
   if (pairs > sm_count / 2) pairs = sm_count / 2;
-  if (pairs < 1) {   // a single SM: plain launch
-    kernel<<<(unsigned)(ntiles < sm_count ? ntiles : sm_count), threads, smem, stream>>>(a, maps);
-    return cudaGetLastError();
-  }
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)(2 * pairs));
-  cfg.blockDim = dim3((unsigned)threads);
-  cfg.dynamicSmemBytes = smem;
-  cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = 2;
-  attr[0].val.clusterDim.y = 1;
-  attr[0].val.clusterDim.z = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, a, maps);
+  if (pairs < 1)   // a single SM: no pairs
+    return launch_dependent(kernel, (unsigned)(ntiles < sm_count ? ntiles : sm_count), threads, smem, stream, 1, a, maps);
+  cudaError_t e = launch_dependent(kernel, (unsigned)(2 * pairs), threads, smem, stream, 2, a, maps);
   if (e == cudaSuccess) return e;
   // a device that cannot co-schedule the pairs: the same kernel without clusters
   cudaGetLastError();
   const int64_t grid = ntiles < sm_count ? ntiles : sm_count;
-  kernel<<<(unsigned)grid, threads, smem, stream>>>(a, maps);
-  return cudaGetLastError();
+  return launch_dependent(kernel, (unsigned)grid, threads, smem, stream, 1, a, maps);
 }
 
 template <int NTP, bool HAS_E, bool HAS_P>
@@ -330,6 +315,7 @@ codec_umma_project_kernel(const MmaArgs a, const __grid_constant__ UmmaMaps maps
   constexpr int kETile = 1, kPTile = HAS_E ? 2 : 1;   // order of the tiles inside a stage
   constexpr int S = Cfg::kStagesN;
   extern __shared__ __align__(128) unsigned char smem_raw[];
+  asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory");   // the next kernel may set up behind this one
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int nstage1 = a.d / kUmmaCols;                                  // stages of one matrix
   const int nstage = (!HAS_E && !HAS_P && a.src2 != nullptr) ? 2 * nstage1 : nstage1;
@@ -431,6 +417,8 @@ codec_umma_project_kernel(const MmaArgs a, const __grid_constant__ UmmaMaps maps
   asm volatile("barrier.cluster.arrive.release.aligned;\nbarrier.cluster.wait.acquire.aligned;\n" ::: "memory");
   asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
   const uint32_t tmem_base = *tmem_slot_ptr;
+  // set-up done; nothing in global memory is touched before the kernel in front has completed
+  asm volatile("griddepcontrol.wait;\n" ::: "memory");
   bool dead = false;
   auto timed_out = [&]() {
     dead = true;

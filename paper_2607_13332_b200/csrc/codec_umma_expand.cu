@@ -18,11 +18,11 @@ cudaError_t launch_umma_expand_one(const MmaArgs &a, const ExpandGeometry &geo, 
   }
   const int64_t units = geo.ntiles * (a.d / kChunkCols);     // (tile, chunk) pairs, dealt evenly
   int64_t grid = units < sm_count ? units : sm_count;
-  kernel<<<(unsigned)grid, kExpandThreads, smem, stream>>>(a, geo, maps);
+  const cudaError_t launched = launch_dependent(kernel, (unsigned)grid, kExpandThreads, smem, stream, 1, a, geo, maps);
   note_kernel(SSN_KERNEL_UMMA_EXPAND, (HAS_E ? SSN_KVAR_E : 0) | (HAS_P ? SSN_KVAR_P : 0) | (KG == 2 ? SSN_KVAR_WIDE : 0) |
                                           (geo.grid_mode ? SSN_KVAR_ALT : 0) | (a.rowsumsq != nullptr ? SSN_KVAR_ROWSUMSQ : 0) |
                                           (PROWS != kGridPos ? SSN_KVAR_FEWSEQ : 0) | (a.zin2 != nullptr ? SSN_KVAR_TWO_RUNS : 0));
-  return cudaGetLastError();
+  return launched;
 }
 
 }  // namespace

@@ -124,6 +124,7 @@ codec_umma_expand_kernel(const MmaArgs a, const ExpandGeometry geo, const __grid
   const int gpos = PROWS == kGridPos ? kGridPos : geo.gpos, gseqs = PROWS == kGridPos ? kGridSeqs : geo.gseqs;
   constexpr int SU = Cfg::kUStages, SE = Cfg::SE;
   extern __shared__ __align__(128) unsigned char smem_raw[];
+  asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory");   // the next kernel may set up behind this one
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int nchunks = a.d / kChunkCols;
   const int ksteps = (a.k + 15) / 16;
@@ -204,6 +205,8 @@ codec_umma_expand_kernel(const MmaArgs a, const ExpandGeometry geo, const __grid
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
   const uint32_t tmem_base = *tmem_slot_ptr;
+  // set-up done; nothing in global memory is touched before the kernel in front has completed
+  asm volatile("griddepcontrol.wait;\n" ::: "memory");
   bool dead = false;
   auto timed_out = [&]() {
     dead = true;

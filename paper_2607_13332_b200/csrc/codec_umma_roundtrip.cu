@@ -16,9 +16,9 @@ cudaError_t launch_roundtrip_ntp(const MmaArgs &a, const UmmaRoundTripMaps &maps
   }
   int64_t grid = maps.tile_start[maps.count];
   if (grid > sm_count) grid = sm_count;
-  kernel<<<(unsigned)grid, kRoundTripThreads, smem, stream>>>(a, maps);
+  const cudaError_t launched = launch_dependent(kernel, (unsigned)grid, kRoundTripThreads, smem, stream, 1, a, maps);
   note_kernel(SSN_KERNEL_UMMA_ROUNDTRIP, (NTP > 8 ? SSN_KVAR_WIDE : 0) | (LEFT ? SSN_KVAR_ALT : 0));
-  return cudaGetLastError();
+  return launched;
 }
 }  // namespace
 

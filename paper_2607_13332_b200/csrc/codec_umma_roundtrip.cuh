@@ -111,6 +111,7 @@ codec_umma_roundtrip_kernel(const MmaArgs a, const __grid_constant__ UmmaRoundTr
   using Cfg = UmmaRoundTripConfig<NTP>;
   constexpr int S = Cfg::kStagesN, S2 = Cfg::kU2Stages;
   extern __shared__ __align__(128) unsigned char smem_raw[];
+  asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory");   // the next kernel may set up behind this one
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int nstage = (a.B1 != nullptr ? a.d1 : a.d) / kUmmaCols;   // pass 1 runs over the columns of the source
   const int nchunks = a.d / kChunkCols;
@@ -166,6 +167,8 @@ codec_umma_roundtrip_kernel(const MmaArgs a, const __grid_constant__ UmmaRoundTr
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory");
   const uint32_t tmem_base = *tmem_slot_ptr;
+  // set-up done; nothing in global memory is touched before the kernel in front has completed
+  asm volatile("griddepcontrol.wait;\n" ::: "memory");
   bool dead = false;
   auto timed_out = [&]() {
     dead = true;
