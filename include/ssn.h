@@ -41,6 +41,11 @@
  *     filled on first use with atomic updates, so calls may come from several host threads and
  *     for several devices (the current device of the calling thread is used, as for any
  *     runtime call).  The diagnostics ssn_launch_count and ssn_last_kernel are informational.
+ *   - Stream order: a call's work is ordered after everything enqueued on its stream before it,
+ *     as for any kernel launch.  The tensor-core kernels of two consecutive calls may overlap the
+ *     SET-UP of the later one (its barriers and tensor memory, nothing in global memory) with the
+ *     tail of the earlier one (programmatic dependent launch); what either reads or writes is as
+ *     if the calls ran one after the other.
  *   - bf16 buffers whose pointers are 16-byte aligned and whose leading dimensions are
  *     multiples of 8 take the vectorised tensor-core kernels; anything else (fp32, odd
  *     leading dimensions, unaligned views) is still computed, by slower general kernels.
